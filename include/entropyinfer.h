@@ -142,7 +142,15 @@ typedef enum ei_flags {
      for a key block, that block's P.V product is not issued either.  It would add exactly nothing, so the
      output is bit-identical; EI_ITEM_STATS counts the products left out.  Off by default so that the tensor-core
      work of a launch does not depend on the data.                                                          */
-  EI_FLAG_ATTN_SKIP_ZERO_PV = 1u << 9
+  EI_FLAG_ATTN_SKIP_ZERO_PV = 1u << 9,
+  /* Attention by the quad-layout kernels (head_dim 128, block_len 128, segments a multiple of 256): sixteen
+     softmax warps, each owning sixteen query rows and all 128 key columns of a block through the 16-lane
+     tensor-memory shapes, so that the row maximum needs only two shuffles inside a quad of threads and no
+     exchange between warps; per-item records (list offset, visible and masked block counts) are worked out
+     once per plan.  Same tolerances; within a few per cent of the default kernel either way.  Combined with
+     EI_FLAG_ATTN_PERSISTENT: one CTA per SM with a scheduler warp and a ring of item records; combined with
+     EI_FLAG_ATTN_SINGLE_TILE: one 128-row tile per CTA, two CTAs per SM.                                   */
+  EI_FLAG_ATTN_QUAD = 1u << 10
 } ei_flags;
 
 /* Fills *p with the paper's constants (e_t 1e-5, alpha 0.5, delta_t 0.4, cap 3, B_h 2048,
@@ -272,6 +280,18 @@ int ei_plan_set_lengths(ei_plan_t* plan, int seq_len, int q_len, int k_blocks_va
    then clears it.                                                                              */
 int ei_plan_status(ei_plan_t* plan, void* stream);
 
+/* Testing aid for the error contract above (EI_ERR_DEVICE_TIMEOUT): every device-side wait of the library is
+   bounded (2^30 clocks, about half a second) and a wait that runs out sets the plan's status word, after which
+   every later wait returns at once, the kernels run to their common end, wait for their own copies in flight,
+   free their tensor memory and return.  This call makes that path reachable without a faulty GPU:
+   wait_limit_log2 > 0 shortens the bound of the plan's kernels to 2^wait_limit_log2 clocks (0: the default),
+   and skip_ring_item >= 0 makes the producer warp of the default stage-4 kernel (head_dim 128, block_len 128,
+   segments a multiple of 256) leave out that K/V load of every tile pair (item 2j is K of the j-th listed
+   block, 2j + 1 its V; -1: none), so that the consumer's wait for it runs out.  ei_plan_status then reports
+   the timeout and clears it; after ei_plan_debug_waits(plan, 0, -1, stream) the plan works as before.
+   Host-synchronous on `stream`.  No counterpart in the paper.                                             */
+int ei_plan_debug_waits(ei_plan_t* plan, int wait_limit_log2, int skip_ring_item, void* stream);
+
 /* Configured total T (TOTAL mode) or the list capacity (BASE mode).                          */
 int64_t ei_plan_total_blocks(const ei_plan_t* plan);
 /* Number of kernels this library has launched for the plan so far.                           */
@@ -316,8 +336,9 @@ int ei_latent_compress(const ei_compress_params* params, const void* q_window, c
    EI_NOALLOC_SCRATCH_BYTES (32 MiB) that every context loading this library holds until exit.
    Shapes needing more return EI_ERR_SCRATCH_TOO_SMALL (the 128k Llama-3-8B and Llama-3.1-70B
    layers fit).  No cudaMalloc, cudaFree or other allocating routine is called.
-   The first call on a device looks up the array's device address (cudaGetSymbolAddress); make
-   that first call outside any stream capture.  All calls share the one array and it keeps the
+   The first call on a device looks up the array's device address (cudaGetSymbolAddress) and the
+   device's architecture (EI_ERR_ARCH unless sm_100, as ei_plan_create reports it); make that first
+   call outside any stream capture.  All calls share the one array and it keeps the
    previous call's contents (none of which is read before being rewritten): two calls whose
    kernels overlap on the GPU (different streams, or threads) race.  Asynchronous on `stream`.  */
 int ei_entropy_noalloc(const ei_params* params, const void* q, const void* k, float* entropy_out,

@@ -23,6 +23,7 @@ from .binding import (  # noqa: F401
     FLAG_ATTN_PER_CTA,
     FLAG_ATTN_NO_SKIP,
     FLAG_ATTN_SKIP_ZERO_PV,
+    FLAG_ATTN_QUAD,
     ROPE_NO_POOL,
     entropy_noalloc,
     lib,

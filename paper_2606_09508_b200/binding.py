@@ -54,6 +54,7 @@ FLAG_ATTN_PERSISTENT = 64
 FLAG_ATTN_PER_CTA = 128
 FLAG_ATTN_NO_SKIP = 256
 FLAG_ATTN_SKIP_ZERO_PV = 512
+FLAG_ATTN_QUAD = 1024
 
 # every symbol the header declares: (name, restype, argtypes)
 _P = C.c_void_p
@@ -77,6 +78,7 @@ SYMBOLS = [
     ("ei_plan_set_lists", C.c_int, [_P, _P, _P, C.c_size_t, _P]),
     ("ei_plan_set_lengths", C.c_int, [_P, C.c_int, C.c_int, C.c_int]),
     ("ei_plan_status", C.c_int, [_P, _P]),
+    ("ei_plan_debug_waits", C.c_int, [_P, C.c_int, C.c_int, _P]),
     ("ei_plan_total_blocks", C.c_int64, [_P]),
     ("ei_plan_launches", C.c_int64, [_P]),
     ("ei_entropy_noalloc", C.c_int, [C.POINTER(EiParams), _P, _P, _P, _P]),
@@ -311,6 +313,11 @@ class Plan:
 
     def status(self, stream=None) -> int:
         return lib().ei_plan_status(self._h, _stream_ptr(stream))
+
+    def debug_waits(self, wait_limit_log2: int = 0, skip_ring_item: int = -1, stream=None):
+        """Testing aid: shorten the device-side wait bound and / or make the producer leave out one K/V load."""
+        _check(lib().ei_plan_debug_waits(self._h, int(wait_limit_log2), int(skip_ring_item), _stream_ptr(stream)),
+               "ei_plan_debug_waits")
 
     def total_blocks(self) -> int:
         return lib().ei_plan_total_blocks(self._h)

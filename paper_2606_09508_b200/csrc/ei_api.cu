@@ -36,6 +36,8 @@ struct ei_plan_s {
   ei::Stats* stats;
   int* status;
   int* sched;  // item counter of the persistent attention kernel
+  int* items;  // per (list cell, tile pair) records for stage 4, rebuilt when the lists change
+  bool items_valid;
   int device;  // the device the plan's storage lives on
   // host-path staging
   __nv_bfloat16 *sq, *sk, *sv, *so;
@@ -238,7 +240,7 @@ void ei_plan_destroy(ei_plan_t* pl) {
   if (!pl) return;
   void* ptrs[] = {pl->entropy, pl->rigid, pl->Mfx, pl->kblocks, pl->offsets, pl->indices, pl->scores, pl->qmax,
                   pl->qmin, pl->kmax, pl->kmin, pl->stats, pl->status, pl->sq, pl->sk, pl->sv, pl->so,
-                  pl->g_entropy, pl->g_scores, pl->sched};
+                  pl->g_entropy, pl->g_scores, pl->sched, pl->items};
   for (void* p : ptrs)
     if (p) cudaFree(p);
   for (int g = 0; pl->sub && g < pl->shape.Hkv; ++g)
@@ -293,13 +295,13 @@ int ei_plan_create(const ei_params* params, ei_plan_t** out) {
             (!pl->group || (dalloc(&pl->g_entropy, (size_t)ls.cells) && dalloc(&pl->g_scores, (size_t)lall))) &&
             dalloc(&pl->scores, (size_t)all) && dalloc(&pl->qmax, (size_t)s.cells * s.d) &&
             dalloc(&pl->qmin, (size_t)s.cells * s.d) && dalloc(&pl->kmax, (size_t)s.Hkv * s.C_B * s.d) &&
-            dalloc(&pl->kmin, (size_t)s.Hkv * s.C_B * s.d) && dalloc(&pl->stats, 1) && dalloc(&pl->status, 1) &&
-            dalloc(&pl->sched, 2);
+            dalloc(&pl->kmin, (size_t)s.Hkv * s.C_B * s.d) && dalloc(&pl->stats, 1) && dalloc(&pl->status, 4) &&
+            dalloc(&pl->sched, 2) && dalloc(&pl->items, (size_t)ls.cells * (s.L_S >= 256 ? s.L_S / 256 : 1) * 8);
   if (!ok) {
     ei_plan_destroy(pl);
     return EI_ERR_ALLOC;
   }
-  if (cudaMemset(pl->status, 0, sizeof(int)) != cudaSuccess || cudaMemset(pl->sched, 0, 2 * sizeof(int)) != cudaSuccess || cudaMemset(pl->stats, 0, sizeof(ei::Stats)) != cudaSuccess) {
+  if (cudaMemset(pl->status, 0, 4 * sizeof(int)) != cudaSuccess || cudaMemset(pl->sched, 0, 2 * sizeof(int)) != cudaSuccess || cudaMemset(pl->stats, 0, sizeof(ei::Stats)) != cudaSuccess) {
     ei_plan_destroy(pl);
     return EI_ERR_CUDA;
   }
@@ -353,7 +355,10 @@ int ei_stage_select(ei_plan_t* pl, void* stream) {
   cudaError_t e = ei::launch_select(pl->lshape, pl->group ? pl->g_scores : pl->scores, pl->kblocks, pl->offsets,
                                     pl->indices, (cudaStream_t)stream);
   pl->launches += 1;
-  if (e == cudaSuccess) pl->planned = true;
+  if (e == cudaSuccess) {
+    pl->planned = true;
+    pl->items_valid = false;
+  }
   return e == cudaSuccess ? EI_OK : EI_ERR_CUDA;
 }
 
@@ -437,6 +442,16 @@ static int attend(ei_plan_t* pl, const void* q, const void* k, const void* v, vo
   a.single_tile = (pl->params.flags & EI_FLAG_ATTN_SINGLE_TILE) != 0;
   a.pair_8warp = (pl->params.flags & EI_FLAG_ATTN_PAIR_8WARP) != 0;
   a.persistent = (pl->params.flags & EI_FLAG_ATTN_PERSISTENT) != 0;
+  a.quad_kernel = (pl->params.flags & EI_FLAG_ATTN_QUAD) != 0;
+  a.items = nullptr;
+  if (a.quad_kernel && full.L_S % 256 == 0) {
+    if (!pl->items_valid) {  // the lists changed since the records were made
+      if (ei::launch_attention_items(pl->lshape, pl->offsets, pl->indices, pl->items, st) != cudaSuccess) return EI_ERR_CUDA;
+      pl->items_valid = true;
+      pl->launches += 1;
+    }
+    a.items = pl->items + (h0 / full.list_div) * full.C_S * (full.L_S / 256) * 8;
+  }
   a.sched = pl->sched;
   a.skip_log2 = (pl->params.flags & EI_FLAG_ATTN_NO_SKIP) ? INFINITY : 24.0f;
   a.pv_skipped = (pl->params.flags & EI_FLAG_ATTN_SKIP_ZERO_PV) ? &pl->stats->pv_skipped : nullptr;
@@ -532,7 +547,7 @@ int ei_prefill_host(ei_plan_t* pl, const void* qh, const void* kh, const void* v
            cudaMemcpyAsync(pl->sv + g * v_head, (const __nv_bfloat16*)vh + g * v_head, v_head * 2,
                            cudaMemcpyHostToDevice, pl->up) == cudaSuccess &&
            cudaEventRecord(ev_v[g], pl->up) == cudaSuccess;
-    if (!ok) return EI_ERR_CUDA;
+    if (!ok) rc = EI_ERR_CUDA;  // (falls through to the join below: copies already queued must not outlive the call)
     for (int g = 0; rc == EI_OK && g < s.Hkv; ++g) {
       ei_plan_t* sb = pl->sub[g];
       const __nv_bfloat16 *qg = pl->sq + g * o_group, *kg = pl->sk + g * k_head, *vg = pl->sv + g * v_head;
@@ -555,9 +570,8 @@ int ei_prefill_host(ei_plan_t* pl, const void* qh, const void* kh, const void* v
       ok = cudaMemcpyAsync(pl->sv + g * v_head, (const __nv_bfloat16*)vh + g * v_head, v_head * 2, cudaMemcpyHostToDevice,
                            pl->up) == cudaSuccess &&
            cudaEventRecord(ev_v[g], pl->up) == cudaSuccess;
-    if (!ok) return EI_ERR_CUDA;
-    if (cudaStreamWaitEvent(st, ev_kq, 0) != cudaSuccess) return EI_ERR_CUDA;
-    rc = ei_plan(pl, pl->sq, pl->sk, pl->sv, stream);
+    if (!ok || cudaStreamWaitEvent(st, ev_kq, 0) != cudaSuccess) rc = EI_ERR_CUDA;  // (joined below all the same)
+    if (rc == EI_OK) rc = ei_plan(pl, pl->sq, pl->sk, pl->sv, stream);
     for (int g = 0; rc == EI_OK && g < s.Hkv; ++g) {
       if (cudaStreamWaitEvent(st, ev_v[g], 0) != cudaSuccess) rc = EI_ERR_CUDA;
       if (rc == EI_OK) rc = attend(pl, pl->sq, pl->sk, pl->sv, pl->so, g, 1, st);
@@ -574,6 +588,15 @@ int ei_prefill_host(ei_plan_t* pl, const void* qh, const void* kh, const void* v
                       cudaStreamSynchronize(pl->up) == cudaSuccess && cudaStreamSynchronize(st) == cudaSuccess;
   if (rc != EI_OK) return rc;
   return joined ? EI_OK : EI_ERR_CUDA;
+}
+
+int ei_plan_debug_waits(ei_plan_t* pl, int wait_limit_log2, int skip_ring_item, void* stream) {
+  if (!pl || wait_limit_log2 < 0 || wait_limit_log2 >= 40 || skip_ring_item < -1) return EI_ERR_INVALID_ARG;
+  if (!on_plan_device(pl)) return EI_ERR_WRONG_DEVICE;
+  const int v[2] = {wait_limit_log2, skip_ring_item + 1};
+  cudaStream_t st = (cudaStream_t)stream;
+  if (cudaMemcpyAsync(pl->status + 1, v, sizeof(v), cudaMemcpyHostToDevice, st) != cudaSuccess) return EI_ERR_CUDA;
+  return cudaStreamSynchronize(st) == cudaSuccess ? EI_OK : EI_ERR_CUDA;
 }
 
 int ei_plan_get(const ei_plan_t* pl, int item, const void** dev_ptr, size_t* bytes) {
@@ -600,6 +623,7 @@ int ei_plan_write(ei_plan_t* pl, int item, const void* host_src, size_t bytes, v
   if (!it.ptr || bytes > it.bytes) return EI_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   if (cudaMemcpyAsync(it.ptr, host_src, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return EI_ERR_CUDA;
+  pl->items_valid = false;  // the item may be part of the lists
   return cudaStreamSynchronize(st) == cudaSuccess ? EI_OK : EI_ERR_CUDA;
 }
 
@@ -629,6 +653,7 @@ int ei_plan_set_lists(ei_plan_t* pl, const int32_t* k_host, const int32_t* idx_h
     return EI_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return EI_ERR_CUDA;
   pl->planned = true;
+  pl->items_valid = false;
   return EI_OK;
 }
 
@@ -653,6 +678,7 @@ int ei_plan_set_lengths(ei_plan_t* pl, int seq_len, int q_len, int k_blocks_vali
   probe.params = p;
   probe.k_first = k_blocks_valid;
   probe.planned = false;
+  probe.items_valid = false;
   *pl = probe;
   return EI_OK;
 }

@@ -15,7 +15,9 @@
 //
 // Tensor memory: S0 at column 0, S1 at 128, O at 256 (512 columns allocated, one CTA per SM).
 // Every mbarrier wait is bounded; on expiry the CTA records EI_ERR_DEVICE_TIMEOUT in the status
-// word, drains its own TMA loads, frees its tensor memory and returns.
+// word, drains its own TMA loads, frees its tensor memory and returns.  Once the status word is set
+// every later wait (of this and of later CTAs) returns at once, so all threads of a CTA run to the
+// common end without taking another path: there is no early exit that only some warps could take.
 #include <cuda.h>
 
 #include "ei_internal.cuh"
@@ -54,7 +56,6 @@ sparse_attention_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_co
                         int* __restrict__ status, Shape s, float scale_log2) {
   using L = AttSmem<D, BN, NS, P_SMEM>;
   extern __shared__ unsigned char att_smem_raw[];
-  if (*reinterpret_cast<volatile int*>(status) != 0) return;  // an earlier CTA gave up: do nothing
 
   const uint32_t raw = smem_u32(att_smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -141,7 +142,7 @@ sparse_attention_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_co
           tma_load_3d(sK + st * L::KV_BYTES + p * (BN * 128), &tmk, p * 64, blk * BN, g, BAR(B_KFULL + st));
         ok = mbar_wait(BAR(B_VEMPTY + st), ph ^ 1, status);
         if (!ok) {  // the K load above is in flight: wait for it before leaving
-          mbar_wait(BAR(B_KFULL + st), ph, status);
+          mbar_wait_drain(BAR(B_KFULL + st), ph);
           break;
         }
         mbar_expect_tx(BAR(B_VFULL + st), L::KV_BYTES);
@@ -151,10 +152,10 @@ sparse_attention_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_co
         issued = it + 1;
       }
       // Drain: every load this thread issued must have landed before the CTA's shared memory is released.
-      mbar_wait(BAR(B_QFULL), 0, status);
+      mbar_wait_drain(BAR(B_QFULL), 0);
       for (int it = (issued > NS ? issued - NS : 0); it < issued; ++it) {
-        mbar_wait(BAR(B_KFULL + it % NS), (it / NS) & 1, status);
-        mbar_wait(BAR(B_VFULL + it % NS), (it / NS) & 1, status);
+        mbar_wait_drain(BAR(B_KFULL + it % NS), (it / NS) & 1);
+        mbar_wait_drain(BAR(B_VFULL + it % NS), (it / NS) & 1);
       }
     }
   } else if (warp == 5) {
@@ -390,7 +391,6 @@ sparse_attention_pair_kernel(const __grid_constant__ CUtensorMap tmq, const __gr
                              int* __restrict__ status, Shape s, float scale_log2) {
   using L = Att2Smem<D, BN, NSLOT>;
   extern __shared__ unsigned char att_smem_raw[];
-  if (*reinterpret_cast<volatile int*>(status) != 0) return;
 
   const uint32_t raw = smem_u32(att_smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -483,10 +483,10 @@ sparse_attention_pair_kernel(const __grid_constant__ CUtensorMap tmq, const __gr
         issued = u + 1;
       }
       // Drain: every load issued here must have landed before the CTA's shared memory is released.
-      mbar_wait(BAR(B_QFULL), 0, status);
-      mbar_wait(BAR(B_QFULL + 1), 0, status);
+      mbar_wait_drain(BAR(B_QFULL), 0);
+      mbar_wait_drain(BAR(B_QFULL + 1), 0);
       for (int u = (issued > NSLOT ? issued - NSLOT : 0); u < issued; ++u)
-        mbar_wait(BAR(B_FULL + u % NSLOT), (u / NSLOT) & 1, status);
+        mbar_wait_drain(BAR(B_FULL + u % NSLOT), (u / NSLOT) & 1);
     }
   } else if (warp == 9) {
     // ================= MMA issuer (whole warp, elected lane issues) =================
@@ -775,7 +775,6 @@ sparse_attention_split_kernel(const __grid_constant__ CUtensorMap tmq, const __g
   static_assert(BN == 128, "the split-row kernel is written for 128-wide key blocks");
   constexpr int OH = D / 2;   // O columns per softmax thread
   extern __shared__ unsigned char att_smem_raw[];
-  if (*reinterpret_cast<volatile int*>(status) != 0) return;
 
   const uint32_t raw = smem_u32(att_smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -850,9 +849,11 @@ sparse_attention_split_kernel(const __grid_constant__ CUtensorMap tmq, const __g
       tma_load_3d(sRing + slot * L::KV_BYTES + p * (BN * 128), tm, p * 64, blk * BN, g, BAR(B_FULL + slot));
   };
   int issued = 0;
+  // testing aid (ei_plan_debug_waits): one ring item the producer leaves out, so that a bounded wait runs out
+  const int skip_item = warp == 16 ? reinterpret_cast<volatile int*>(status)[2] - 1 : -1;
   if (warp == 16 && n1 > 0) {
     for (int u = 0; u < 2 * n1 && u < NSLOT; ++u) {
-      load_item(u, __ldg(indices + off + (u >> 1)));
+      if (u != skip_item) load_item(u, __ldg(indices + off + (u >> 1)));
       issued = u + 1;
     }
     tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), TM_COLS);
@@ -868,8 +869,8 @@ sparse_attention_split_kernel(const __grid_constant__ CUtensorMap tmq, const __g
       for (int c = 0; c < D / 8; ++c) reinterpret_cast<uint4*>(orow)[c] = make_uint4(0, 0, 0, 0);
     }
     if (warp == 16) {  // the Q loads are in flight: let them land before the CTA goes away
-      mbar_wait(BAR(B_QFULL), 0, status);
-      mbar_wait(BAR(B_QFULL + 1), 0, status);
+      mbar_wait_drain(BAR(B_QFULL), 0);
+      mbar_wait_drain(BAR(B_QFULL + 1), 0);
     }
     return;
   }
@@ -886,15 +887,15 @@ sparse_attention_split_kernel(const __grid_constant__ CUtensorMap tmq, const __g
       const int blk_next = ((u & 1) && (u >> 1) + 1 < n1) ? __ldg(indices + off + (u >> 1) + 1) : blk;
       ok = mbar_wait(BAR(B_EMPTY + slot), ph ^ 1, status);
       if (!ok) break;
-      load_item(u, blk);
+      if (u != skip_item) load_item(u, blk);
       issued = u + 1;
       blk = blk_next;
     }
     // Drain: every load issued here must have landed before the CTA's shared memory is released.
-    mbar_wait(BAR(B_QFULL), 0, status);
-    mbar_wait(BAR(B_QFULL + 1), 0, status);
+    mbar_wait_drain(BAR(B_QFULL), 0);
+    mbar_wait_drain(BAR(B_QFULL + 1), 0);
     for (int u = (issued > NSLOT ? issued - NSLOT : 0); u < issued; ++u)
-      mbar_wait(BAR(B_FULL + u % NSLOT), (u / NSLOT) & 1, status);
+      if (u != skip_item) mbar_wait_drain(BAR(B_FULL + u % NSLOT), (u / NSLOT) & 1);
   } else if (warp == 17) {
     // ================= MMA issuer (whole warp, elected lane issues) =================
     constexpr uint32_t IDESC_QK = make_idesc(BN, false);
@@ -1251,7 +1252,8 @@ sparse_attention_persistent_kernel(const __grid_constant__ CUtensorMap tmq, cons
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const bool dead = *reinterpret_cast<volatile int*>(status) != 0;  // an earlier launch gave up: take no work
+  // an earlier launch gave up: take no work (one answer per warp, whatever the lanes read)
+  const bool dead = __any_sync(0xffffffffu, *reinterpret_cast<volatile int*>(status) != 0);
 
   bool ok = true;
   const int pairs_per_seg = s.L_S / (2 * BM);
@@ -1335,11 +1337,11 @@ sparse_attention_persistent_kernel(const __grid_constant__ CUtensorMap tmq, cons
     }
     // Drain: every load issued here must have landed before the CTA's shared memory is released.
     if (last_q >= 0) {
-      mbar_wait(BAR(B_QFULL), last_q & 1, status);
-      mbar_wait(BAR(B_QFULL + 1), last_q & 1, status);
+      mbar_wait_drain(BAR(B_QFULL), last_q & 1);
+      mbar_wait_drain(BAR(B_QFULL + 1), last_q & 1);
     }
     for (int u = (ucount > NSLOT ? ucount - NSLOT : 0); u < ucount; ++u)
-      mbar_wait(BAR(B_FULL + u % NSLOT), (u / NSLOT) & 1, status);
+      mbar_wait_drain(BAR(B_FULL + u % NSLOT), (u / NSLOT) & 1);
   } else if (warp == 17) {
     // ================= MMA issuer =================
     constexpr uint32_t IDESC_QK = make_idesc(BN, false);
@@ -1653,7 +1655,7 @@ static EncodeTiledFn get_encode_fn() {
 }
 
 // bf16 tensor [heads, N, d] (d contiguous) viewed as a 3-D map, box = 64 x rows x 1, 128-byte swizzle
-static bool make_map(CUtensorMap* tm, const void* ptr, int d, int N, int heads, int64_t tok_stride,
+bool make_tensor_map(CUtensorMap* tm, const void* ptr, int d, int N, int heads, int64_t tok_stride,
                      int64_t head_stride, int box_rows) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
@@ -1672,9 +1674,9 @@ static int launch_t(const Shape& s, const AttnArgs& a, cudaStream_t st) {
   using L = AttSmem<D, BN, NS, P_SMEM>;
   static_assert(L::DYN_BYTES <= 232448, "shared memory budget exceeded");
   CUtensorMap tmq, tmk, tmv;
-  if (!make_map(&tmq, a.q, D, s.Nq, s.H, s.qs_t, s.qs_h, BM) ||
-      !make_map(&tmk, a.k, D, s.N, s.Hkv, s.ks_t, s.ks_h, BN) ||
-      !make_map(&tmv, a.v, D, s.N, s.Hkv, s.vs_t, s.vs_h, BN))
+  if (!make_tensor_map(&tmq, a.q, D, s.Nq, s.H, s.qs_t, s.qs_h, BM) ||
+      !make_tensor_map(&tmk, a.k, D, s.N, s.Hkv, s.ks_t, s.ks_h, BN) ||
+      !make_tensor_map(&tmv, a.v, D, s.N, s.Hkv, s.vs_t, s.vs_h, BN))
     return EI_ERR_CUDA;
   auto kern = sparse_attention_kernel<D, BN, NS, P_SMEM>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES) != cudaSuccess)
@@ -1691,9 +1693,9 @@ static int launch_pair_t(const Shape& s, const AttnArgs& a, cudaStream_t st) {
   using L = Att2Smem<D, BN, NSLOT>;
   static_assert(L::DYN_BYTES <= 232448, "shared memory budget exceeded");
   CUtensorMap tmq, tmk, tmv;
-  if (!make_map(&tmq, a.q, D, s.Nq, s.H, s.qs_t, s.qs_h, BM) ||
-      !make_map(&tmk, a.k, D, s.N, s.Hkv, s.ks_t, s.ks_h, BN) ||
-      !make_map(&tmv, a.v, D, s.N, s.Hkv, s.vs_t, s.vs_h, BN))
+  if (!make_tensor_map(&tmq, a.q, D, s.Nq, s.H, s.qs_t, s.qs_h, BM) ||
+      !make_tensor_map(&tmk, a.k, D, s.N, s.Hkv, s.ks_t, s.ks_h, BN) ||
+      !make_tensor_map(&tmv, a.v, D, s.N, s.Hkv, s.vs_t, s.vs_h, BN))
     return EI_ERR_CUDA;
   auto kern = sparse_attention_pair_kernel<D, BN, NSLOT>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES) != cudaSuccess)
@@ -1710,9 +1712,9 @@ static int launch_split_t(const Shape& s, const AttnArgs& a, cudaStream_t st) {
   using L = Att3Smem<D, BN, NSLOT>;
   static_assert(L::DYN_BYTES <= 232448, "shared memory budget exceeded");
   CUtensorMap tmq, tmk, tmv;
-  if (!make_map(&tmq, a.q, D, s.Nq, s.H, s.qs_t, s.qs_h, BM) ||
-      !make_map(&tmk, a.k, D, s.N, s.Hkv, s.ks_t, s.ks_h, BN) ||
-      !make_map(&tmv, a.v, D, s.N, s.Hkv, s.vs_t, s.vs_h, BN))
+  if (!make_tensor_map(&tmq, a.q, D, s.Nq, s.H, s.qs_t, s.qs_h, BM) ||
+      !make_tensor_map(&tmk, a.k, D, s.N, s.Hkv, s.ks_t, s.ks_h, BN) ||
+      !make_tensor_map(&tmv, a.v, D, s.N, s.Hkv, s.vs_t, s.vs_h, BN))
     return EI_ERR_CUDA;
   auto kern = sparse_attention_split_kernel<D, BN, NSLOT>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES) != cudaSuccess)
@@ -1729,9 +1731,9 @@ static int launch_persistent_t(const Shape& s, const AttnArgs& a, cudaStream_t s
   using L = Att4Smem<D, BN, NSLOT>;
   static_assert(L::DYN_BYTES <= 232448, "shared memory budget exceeded");
   CUtensorMap tmq, tmk, tmv;
-  if (!make_map(&tmq, a.q, D, s.Nq, s.H, s.qs_t, s.qs_h, BM) ||
-      !make_map(&tmk, a.k, D, s.N, s.Hkv, s.ks_t, s.ks_h, BN) ||
-      !make_map(&tmv, a.v, D, s.N, s.Hkv, s.vs_t, s.vs_h, BN))
+  if (!make_tensor_map(&tmq, a.q, D, s.Nq, s.H, s.qs_t, s.qs_h, BM) ||
+      !make_tensor_map(&tmk, a.k, D, s.N, s.Hkv, s.ks_t, s.ks_h, BN) ||
+      !make_tensor_map(&tmv, a.v, D, s.N, s.Hkv, s.vs_t, s.vs_h, BN))
     return EI_ERR_CUDA;
   auto kern = sparse_attention_persistent_kernel<D, BN, NSLOT>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES) != cudaSuccess)
@@ -1752,6 +1754,7 @@ int launch_attention(const Shape& s, const AttnArgs& a, cudaStream_t st) {
     if (s.L_B == 64) return launch_t<256, 64, 2, false>(s, a, st);
     return EI_ERR_UNSUPPORTED_SHAPE;
   }
+  if (a.quad_kernel && s.L_S % (2 * BM) == 0 && s.d == 128 && s.L_B == 128) return launch_attention_quad(s, a, st);
   if (a.persistent && a.sched && s.L_S % (2 * BM) == 0 && s.d == 128 && s.L_B == 128)
     return launch_persistent_t<128, 128, 5>(s, a, st);
 

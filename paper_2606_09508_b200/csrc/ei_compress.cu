@@ -444,6 +444,8 @@ __global__ void __launch_bounds__(TOPK_THREADS, 1) topk_cluster_kernel(const flo
       const int j = p0 + u * 32 + lane;
       if (j < L) out[j] = j;
     }
+    chain_wait();  // every link of the chain waits for the one before it, so that whatever follows this grid is
+                   // also ordered after the scoring kernel's writes (w and its histogram)
     return;
   }
   for (int x = tid; x < 3 * 256; x += TOPK_THREADS) (&hist[0][0])[x] = 0;

@@ -1,6 +1,7 @@
 // Internal declarations shared by the CUDA translation units of libentropyinfer.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -93,12 +94,22 @@ struct AttnArgs {
   bool single_tile;  // force the one-tile-per-CTA kernel
   bool pair_8warp;   // force the two-tile kernel with one softmax thread per row
   bool persistent;   // the persistent form of the split-row kernel (items off a counter)
+  bool quad_kernel;  // the quad-layout kernel (ei_attention_quad.cu)
   int* sched;        // two ints, zero between launches: next item, CTAs finished
   float skip_log2;   // split-row kernels: half rows more than this many binary orders below the row maximum get P = 0
                      // without being exponentiated (infinity: never)
   long long* pv_skipped;  // device counter: (tile, block) P.V products left out because P was all zero (may be null)
+  const int* items;       // per (list cell, tile pair) records of launch_attention_items (quad-layout kernels), shifted like offsets
 };
 // returns EI_OK or a negative ei_status (tensor-map encoding can fail)
 int launch_attention(const Shape& s, const AttnArgs& a, cudaStream_t st);
+int launch_attention_quad(const Shape& s, const AttnArgs& a, cudaStream_t st);  // d = 128, L_B = 128, L_S % 256 = 0
+// one record of 8 ints per (list cell, tile pair) from the plan's lists (ls: the list-head shape); a no-op for
+// shapes the tile-pair kernels do not take
+cudaError_t launch_attention_items(const Shape& ls, const int* offsets, const int* indices, int* items, cudaStream_t st);
+
+// bf16 tensor [heads, N, d] (d contiguous) as a 3-D tensor map, box = 64 x box_rows x 1, 128-byte swizzle
+bool make_tensor_map(CUtensorMap* tm, const void* ptr, int d, int N, int heads, int64_t tok_stride,
+                     int64_t head_stride, int box_rows);
 
 }  // namespace ei

@@ -28,6 +28,10 @@ int scratch_for_current_device(unsigned char** out) {
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return EI_ERR_CUDA;
   std::lock_guard<std::mutex> lock(g_mu);
   if (!g_scratch_ptr[dev]) {
+    // the kernels are built for sm_100 only: say so, as ei_plan_create does, instead of failing in a launch
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return EI_ERR_CUDA;
+    if (major != 10) return EI_ERR_ARCH;
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, ei_noalloc_scratch) != cudaSuccess || !p) return EI_ERR_CUDA;
     g_scratch_ptr[dev] = static_cast<unsigned char*>(p);

@@ -424,7 +424,8 @@ pool_observe_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
   auto FULL = [&](int b) { return bar0 + 8u * b; };
   auto EMPTY = [&](int b) { return bar0 + 16u + 8u * b; };
 
-  if (*reinterpret_cast<volatile int*>(status) != 0) return;
+  // an earlier wait gave up: do nothing (decided for the whole CTA at once, so no warp is left at a barrier)
+  if (__syncthreads_or(*reinterpret_cast<volatile int*>(status) != 0)) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) {
     for (int b = 0; b < 2; ++b) {

@@ -83,11 +83,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait: gives up after ~2^30 clocks (about half a second), records the timeout.
+// The status block is four ints: [0] the status code, [1] log2 of the wait limit in clocks when a test has
+// shortened it (0: the default 30), [2] 1 + the K/V ring item the producer is to leave out (0: none; see
+// ei_plan_debug_waits), [3] unused.
 static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, int* status) {
   if (*reinterpret_cast<volatile int*>(status) != 0) return false;  // someone already gave up: do not wait again
+  const int lg = reinterpret_cast<volatile int*>(status)[1];
+  const long long limit = 1LL << (lg > 0 && lg < 40 ? lg : 30);
   const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > (1LL << 30)) {
+    if (clock64() - t0 > limit) {
       atomicExch(status, (int)EI_ERR_DEVICE_TIMEOUT);
       return false;
     }
@@ -97,6 +102,15 @@ static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status) {
   if (mbar_try_wait(bar, parity)) return true;
   return mbar_wait_slow(bar, parity, status);
+}
+// Drain wait: for loads this thread issued itself, which land within microseconds whatever else went wrong.
+// Unlike mbar_wait it does not give way to a status word that is already set (a CTA that has given up must
+// still not release shared memory with its own TMA loads in flight); bounded at ~2^22 clocks all the same.
+static __device__ __noinline__ void mbar_wait_drain(uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity))
+    if (clock64() - t0 > (1LL << 22)) return;
 }
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, int c2,

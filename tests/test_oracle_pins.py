@@ -247,6 +247,25 @@ def test_total_budgets_brute_force_base_search():
         np.testing.assert_array_equal(k.ravel(), want)
 
 
+def _golden_base_budgets():
+    rows = []
+    with open(os.path.join(GOLDEN, "base_budgets_fixed_point.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            name, r, base, m, k = [s.strip() for s in line.split("|")]
+            rows.append((name, int(r), float(base), [float(x) for x in m.split()], [int(x) for x in k.split()]))
+    return rows
+
+
+@pytest.mark.parametrize("name,r,base_blocks,m,k_want", _golden_base_budgets())
+def test_base_budgets_hand_worked_fixed_point(name, r, base_blocks, m, k_want):
+    # exact: the fixed-point product decides, including where it lands on an integer or one below the real floor
+    k = oracle.budgets_base(np.array([m], np.float64), r, base_blocks)
+    np.testing.assert_array_equal(k[0], k_want)
+
+
 def test_base_budgets_respect_paper_bound():
     # BASE mode: k <= 3 B_h / L_B and executed work sum_i k_i L_B L_S <= 3 B_h N (Eq. t_spa).
     rng = np.random.default_rng(6)

@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2606_09508_b200 as ei
 import synth
 from util import to_dev
@@ -57,6 +58,39 @@ def test_noalloc_entropy_matches_plan_path_twice_in_a_row():
         want = _reference_entropy(wl, qd, kd).astype(np.float64)
         got = out.cpu().numpy().astype(np.float64)
         assert (np.abs(got - want) <= 1e-3 * np.abs(want) + 1e-7).all()
+
+
+def test_noalloc_entropy_against_the_oracle_and_without_allocating():
+    # Not only the same kernels through another door: the table must be the CPU oracle's (fp64, written from the
+    # paper) within the entropy tolerance, also for a chunk of queries (q_len < seq_len).  And the property in the
+    # entry point's name: the device's free memory is the same after the calls as before them (one call first, so
+    # that one-time set-up by the CUDA runtime is not counted).
+    wl = CASES[1]
+    q, k, v, st = synth.generate(wl)
+    qd, kd = to_dev(q), to_dev(k)
+    whole = ei.params_default(wl.H, wl.Hkv, wl.d, wl.N, wl.L_S, wl.L_B, wl.fraction)
+    n_q = wl.N // 2                                   # the second half of the sequence as a chunk
+    chunk = ei.params_default(wl.H, wl.Hkv, wl.d, wl.N, wl.L_S, wl.L_B, wl.fraction)
+    chunk.q_len = n_q
+    chunk.q_stride_head = wl.N * wl.d                 # the chunk's queries sit inside the whole tensor
+    out_w = torch.full((wl.H, wl.C_S), float("nan"), dtype=torch.float32, device="cuda")
+    out_c = torch.full((wl.H, n_q // wl.L_S), float("nan"), dtype=torch.float32, device="cuda")
+    q_chunk = qd[:, wl.N - n_q:, :]
+    ei.entropy_noalloc(whole, qd, kd, out_w)
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    for _ in range(3):
+        ei.entropy_noalloc(whole, qd, kd, out_w)
+        ei.entropy_noalloc(chunk, q_chunk, kd, out_c)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before
+    want_w = oracle.plan(q, k, wl.L_S, wl.L_B, fraction=wl.fraction).entropy64
+    got_w = out_w.cpu().numpy().astype(np.float64)
+    assert (np.abs(got_w - want_w) <= 1e-3 * np.abs(want_w) + 1e-7).all(), np.abs(got_w - want_w).max()
+    want_c = oracle.plan(q[:, wl.N - n_q:], k, wl.L_S, wl.L_B, fraction=wl.fraction).entropy64
+    got_c = out_c.cpu().numpy().astype(np.float64)
+    assert want_c.shape == got_c.shape
+    assert (np.abs(got_c - want_c) <= 1e-3 * np.abs(want_c) + 1e-7).all(), np.abs(got_c - want_c).max()
 
 
 def test_noalloc_rejects_shapes_beyond_the_fixed_scratch():
