@@ -31,11 +31,44 @@ METRIC = "128k-token sparse prefill attention ms/layer; tensor-pipe % of B200 pe
 UNIT = "ms/layer"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 NOMINAL_BF16_TFLOPS = 2250.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from a one-pass ncu capture of this
-# command (see profiles/sparse_attention_split_kernel_llama3_8b.md); None where no capture exists.
-NCU_DRAM_BYTES_PER_LAUNCH = {("llama3_8b_128k", 0.05, "sparse_attention_persistent_kernel"): 3.596e9,
-                             ("llama3_8b_128k", 0.05, "sparse_attention_split_kernel"): 3.585e9,
-                             ("llama3_8b_32k", 0.10, "sparse_attention_split_kernel"): 0.7329e9}
+NOMINAL_HBM_GBS = 8000.0
+NCU_COUNTERS = os.path.join(ROOT, "profiles", "ncu_counters_attention.txt")
+KERNEL_SOURCES = {"sparse_attention_quad_kernel": "ei_attention_quad.cu", "sparse_attention_quad_persistent_kernel": "ei_attention_quad.cu",
+                  "sparse_attention_quad1_kernel": "ei_attention_quad.cu", "sparse_attention_split_kernel": "ei_attention.cu",
+                  "sparse_attention_persistent_kernel": "ei_attention.cu", "sparse_attention_pair_kernel": "ei_attention.cu",
+                  "sparse_attention_kernel": "ei_attention.cu"}
+
+
+def git_blob_hash(path: str) -> str:
+    """What `git hash-object` prints for the file (sha1 of "blob <size>\\0" + contents); no git needed."""
+    import hashlib
+    with open(path, "rb") as f:
+        data = f.read()
+    return hashlib.sha1(b"blob %d\0" % len(data) + data).hexdigest()
+
+
+def ncu_counters(workload: str, fraction: float, kernel: str, no_skip: bool):
+    """Counters of one ncu capture of this command, from the tracked table profiles/ncu_counters_attention.txt
+    (one row per capture: workload, fraction, kernel, shortcut on/off, the kernel source's git blob hash at
+    capture time, tensor-pipe-active %, DRAM bytes per launch).  A row whose hash is not the current source's is
+    reported as stale and its numbers are withheld."""
+    none = {"tensor_pipe_active_pct_ncu": None, "traffic": None, "stale": None}
+    src = KERNEL_SOURCES.get(kernel)
+    if src is None or not os.path.exists(NCU_COUNTERS):
+        return none
+    cur = git_blob_hash(os.path.join(ROOT, "paper_2606_09508_b200", "csrc", src))
+    with open(NCU_COUNTERS) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if not line:
+                continue
+            wname, frac, kname, mode, h, tp, dram = line.split()
+            if wname == workload and abs(float(frac) - fraction) < 1e-9 and kname == kernel and mode == ("no_skip" if no_skip else "skip"):
+                if h != cur:
+                    return {"tensor_pipe_active_pct_ncu": None, "traffic": None, "stale": True}
+                return {"tensor_pipe_active_pct_ncu": None if tp == "-" else float(tp),
+                        "traffic": None if dram == "-" else float(dram), "stale": False}
+    return none
 
 
 def load_peaks():
@@ -253,10 +286,7 @@ def run_ours(args, wl):
     params = ei.params_default(wl.H, wl.Hkv, wl.d, wl.N, wl.L_S, wl.L_B, wl.fraction)
     if args.group_shared:
         params.flags |= ei.FLAG_GROUP_SHARED
-    if args.attention == "persistent":
-        params.flags |= ei.FLAG_ATTN_PERSISTENT
-    elif args.attention == "per_cta":
-        params.flags |= ei.FLAG_ATTN_PER_CTA
+    params.flags |= attention_flags(ei, args.attention)
     if args.no_skip:
         params.flags |= ei.FLAG_ATTN_NO_SKIP
     plan = ei.Plan(params)
@@ -351,37 +381,36 @@ def run_ours(args, wl):
         every_p = {"attention_ms": ns_ms, "tflops": flops / (ns_ms * 1e-3) / 1e12,
                    "what": "EI_FLAG_ATTN_NO_SKIP: no shortcut for half rows below 2^-24 of the row maximum"}
         del plan2
-        # ... and with the P.V products of all-zero P left out as well (EI_FLAG_ATTN_SKIP_ZERO_PV, bit-identical output)
-        params3 = ei.params_default(wl.H, wl.Hkv, wl.d, wl.N, wl.L_S, wl.L_B, wl.fraction)
-        params3.flags = params.flags | ei.FLAG_ATTN_SKIP_ZERO_PV
-        plan3 = ei.Plan(params3)
-        plan3.plan(qd, kd, vd)
-        out3 = torch.empty_like(out)
-        plan3.sparse_prefill(qd, kd, vd, out3)
-        pv_left_out = int(plan3.read("STATS")[6])
-        plan.plan(qd, kd, vd)
-        plan.sparse_prefill(qd, kd, vd, out)
-        same_bits = bool(torch.equal(out3.view(torch.int16), out.view(torch.int16)))
-        for _ in range(3):
-            plan3.sparse_prefill(qd, kd, vd, out3)
-        ne[0].record(stream)
-        for s_ in range(args.steps):
-            plan3.sparse_prefill(qd, kd, vd, out3)
-            ne[s_ + 1].record(stream)
+    # ---- the same kernel at full budget (every causal block selected): one launch, for the sparse / dense ratio ----
+    dense = None
+    if world == 1 and not args.no_dense:
+        pd = ei.params_default(wl.H, wl.Hkv, wl.d, wl.N, wl.L_S, wl.L_B, 1.0)
+        pd.flags = params.flags
+        pland = ei.Plan(pd)
+        pland.plan(qd, kd, vd)
+        outd = torch.empty_like(out)
+        pland.sparse_prefill(qd, kd, vd, outd)        # warm-up launch
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        d0.record(stream)
+        pland.sparse_prefill(qd, kd, vd, outd)
+        d1.record(stream)
         torch.cuda.synchronize()
-        if plan3.status() != 0:
+        if pland.status() != 0:
             raise RuntimeError("device-side wait timed out")
-        zp_ms = float(np.mean([ne[s_].elapsed_time(ne[s_ + 1]) for s_ in range(args.steps)]))
-        issued_flops = flops - pv_left_out * tile_flops(wl) / 2
-        every_p["zero_pv_left_out"] = {"attention_ms": zp_ms, "pv_products_left_out": pv_left_out, "of": int(tiles),
-                                       "issued_tflop": issued_flops / 1e12,
-                                       "tflops_issued": issued_flops / (zp_ms * 1e-3) / 1e12,
-                                       "bit_identical_to_default": same_bits,
-                                       "what": "EI_FLAG_ATTN_SKIP_ZERO_PV (opt-in)"}
-        del plan3, out3
-        plan.plan(qd, kd, vd)                 # the lists the rest of the run reads are the main plan's again
-        plan.sparse_prefill(qd, kd, vd, out)
-    tensor_peak = peaks["bf16_tflops_sustained"]
+        dres = pland.results()
+        dk = np.repeat(dres["k"], wl.H // wl.Hkv, axis=0) if args.group_shared else dres["k"]
+        dense_ms = d0.elapsed_time(d1)
+        dense = {"attention_ms": dense_ms, "executed_tflop": executed_tiles(wl, dk) * tile_flops(wl) / 1e12,
+                 "tflops": executed_tiles(wl, dk) * tile_flops(wl) / (dense_ms * 1e-3) / 1e12,
+                 "speedup_of_sparse": dense_ms / kernel_ms["attention"], "launches_timed": 1,
+                 "what": "the same stage-4 kernel with every causal block selected (budget 100 %)"}
+        del pland, outd
+    # The tensor roofline's denominator follows the length of the timed region: cuBLAS bf16 as a burst when the
+    # K timed steps take under a second (the clock has not yet come down under the power cap), the seconds-long
+    # sustained figure otherwise.
+    timed_s = ms_per_step * args.steps * 1e-3
+    peak_key = "bf16_tflops" if timed_s < 1.0 else "bf16_tflops_sustained"
+    tensor_peak = peaks[peak_key]
     qk_bytes = (wl.H + wl.Hkv) * wl.N * wl.d * 2
     pool_bytes = qk_bytes + 2 * (wl.H * wl.C_S + wl.Hkv * wl.C_B) * wl.d * 2
     plan_ms = plan_call_ms
@@ -519,7 +548,13 @@ def run_ours(args, wl):
             dist.destroy_process_group()
         return
 
-    traffic = NCU_DRAM_BYTES_PER_LAUNCH.get((wl.name, wl.fraction, attention_kernel_name(wl, args, plan.total_blocks())))
+    kname = attention_kernel_name(wl, args, plan.total_blocks())
+    counters = ncu_counters(wl.name, wl.fraction, kname, args.no_skip)
+    counters_all = ncu_counters(wl.name, wl.fraction, kname, True)
+    if every_p is not None:
+        every_p["frac_of_burst"] = every_p["tflops"] / peaks["bf16_tflops"]
+        every_p["tensor_pipe_active_pct_ncu"] = counters_all["tensor_pipe_active_pct_ncu"]
+        every_p["counters_stale"] = counters_all["stale"]
 
     line = {
         "metric": METRIC, "value": job_value(ms_per_step, world), "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -529,14 +564,19 @@ def run_ours(args, wl):
         "kernel_ms": kernel_ms, "plan_ms": plan_ms, "staged_plan_ms": staged_plan_ms,
         "executed_tiles": tiles, "executed_tflop": flops / 1e12,
         "roofline": {"bound": "tensor", "achieved": att_tflops, "peak": tensor_peak, "unit": "TFLOP/s",
-                     "frac": att_tflops / tensor_peak, "traffic": traffic,
-                     "kernel": attention_kernel_name(wl, args, plan.total_blocks()),
+                     "frac": att_tflops / tensor_peak, "traffic": counters["traffic"],
+                     "kernel": kname,
                      "algorithmic_bytes": int(2 * wl.H * wl.N * wl.d * 2 + 2 * wl.Hkv * wl.N * wl.d * 2),
-                     "tensor_pipe_active_pct_ncu": tensor_pipe_pct(wl, attention_kernel_name(wl, args, plan.total_blocks()), args.no_skip), "peak_kind": f"bf16 sustained, {peaks['source']}",
+                     "tensor_pipe_active_pct_ncu": counters["tensor_pipe_active_pct_ncu"], "stale": counters["stale"],
+                     "peak_kind": f"cuBLAS bf16 {'burst' if peak_key == 'bf16_tflops' else 'sustained'} ({peaks['source']}): "
+                                  f"the {args.steps} timed steps took {timed_s:.2f} s",
                      "frac_of_burst": att_tflops / peaks["bf16_tflops"],
+                     "frac_of_sustained": att_tflops / peaks["bf16_tflops_sustained"],
                      "frac_of_nominal_2250": att_tflops / NOMINAL_BF16_TFLOPS},
+        "dense": dense, "dense_speedup": None if dense is None else dense["speedup_of_sparse"],
         "roofline_plan": {"bound": "hbm", "achieved": qk_bytes / (plan_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
                           "unit": "GB/s", "frac": qk_bytes / (plan_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                          "frac_of_nominal_8000": qk_bytes / (plan_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
                           "what": "Q+K bytes / whole ei_plan call (K pooling, fused Q pooling + observation, budget, select)", "peak_kind": f"copy, {peaks['source']}",
                           "pool_kernel_gbs": pool_bytes / (kernel_ms["pool"] * 1e-3) / 1e9},
         "cuda_graph": graph_info, "group_shared": group_cmp, "every_probability_evaluated": every_p, "latent_compress": compress, "producer_pooling": producer, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
@@ -552,22 +592,23 @@ def run_ours(args, wl):
 # Parameter sweeps (speed only; the paper sweeps segment / block size and budgets for quality, Fig. 5-6, and
 # reports end-to-end latency against input length, Section 5.3).  One JSON line per point.
 # ----------------------------------------------------------------------------------------------
-def tensor_pipe_pct(wl, kernel, no_skip=False):
-    """sm__pipe_tensor_cycles_active (% of elapsed) from the single-pass ncu captures of the benchmark workload
-    (profiles/sparse_attention_split_kernel_llama3_8b.md); None where no capture exists."""
-    if (wl.name, wl.fraction) != ("llama3_8b_128k", 0.05):
-        return None
-    if kernel == "sparse_attention_split_kernel":
-        return 59.54 if no_skip else 67.27
-    return None
+ATTENTION_CHOICES = {"default": "sparse_attention_quad_kernel", "per_cta": "sparse_attention_quad_kernel",
+                     "quad_persistent": "sparse_attention_quad_persistent_kernel",
+                     "quad_single_tile": "sparse_attention_quad1_kernel", "split": "sparse_attention_split_kernel",
+                     "persistent": "sparse_attention_persistent_kernel"}
+
+
+def attention_flags(ei, choice: str) -> int:
+    return {"default": 0, "per_cta": ei.FLAG_ATTN_PER_CTA, "quad_persistent": ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_PERSISTENT,
+            "quad_single_tile": ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_SINGLE_TILE, "split": ei.FLAG_ATTN_SPLIT,
+            "persistent": ei.FLAG_ATTN_PERSISTENT}[choice]
 
 
 def attention_kernel_name(wl, args, total_blocks) -> str:
     """Which stage-4 kernel ei_sparse_prefill launches for this workload."""
-    split_ok = wl.d == 128 and wl.L_B == 128 and wl.L_S % 256 == 0
-    if not split_ok:
+    if not (wl.d == 128 and wl.L_B == 128 and wl.L_S % 256 == 0):
         return "sparse_attention_pair_kernel" if wl.L_S % 256 == 0 else "sparse_attention_kernel"
-    return "sparse_attention_persistent_kernel" if args.attention == "persistent" else "sparse_attention_split_kernel"
+    return ATTENTION_CHOICES[args.attention]
 
 
 def run_chunk_sweep(args, ei, torch, wl):
@@ -659,10 +700,7 @@ def run_sweep(args):
         if mode == "base":
             p.budget_mode = ei.binding.BUDGET_BASE_TOKENS
             p.base_budget_tokens = 2048.0
-        if args.attention == "persistent":
-            p.flags |= ei.FLAG_ATTN_PERSISTENT
-        elif args.attention == "per_cta":
-            p.flags |= ei.FLAG_ATTN_PER_CTA
+        p.flags |= attention_flags(ei, args.attention)
         plan_ms, att_ms, tiles, rigid = timed(p)
         dense = ei.params_default(wl.H, wl.Hkv, wl.d, wl.N, wl.L_S, wl.L_B, 1.0)
         _, dense_att_ms, dense_tiles, _ = timed(dense)
@@ -688,10 +726,11 @@ def main():
     ap.add_argument("--ref-cells", type=int, default=24, help="cells the CPU oracle attends over per step")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-dense", action="store_true", help="skip the one launch at full budget (dense_speedup)")
     ap.add_argument("--with-producer", action="store_true",
                     help="also time the rotary producer with and without the pooling folded in (ei_rope_pool, ei_plan_pooled)")
     ap.add_argument("--with-compress", action="store_true", help="also time the Alg. 4 KV-cache compression")
-    ap.add_argument("--attention", default="default", choices=["default", "persistent", "per_cta"],
+    ap.add_argument("--attention", default="default", choices=sorted(ATTENTION_CHOICES),
                     help="persistent: the persistent form of the two-threads-per-row attention kernel")
     ap.add_argument("--no-skip", action="store_true",
                     help="evaluate every probability (EI_FLAG_ATTN_NO_SKIP): no shortcut for negligible half rows")

@@ -143,14 +143,19 @@ typedef enum ei_flags {
      output is bit-identical; EI_ITEM_STATS counts the products left out.  Off by default so that the tensor-core
      work of a launch does not depend on the data.                                                          */
   EI_FLAG_ATTN_SKIP_ZERO_PV = 1u << 9,
-  /* Attention by the quad-layout kernels (head_dim 128, block_len 128, segments a multiple of 256): sixteen
-     softmax warps, each owning sixteen query rows and all 128 key columns of a block through the 16-lane
-     tensor-memory shapes, so that the row maximum needs only two shuffles inside a quad of threads and no
-     exchange between warps; per-item records (list offset, visible and masked block counts) are worked out
-     once per plan.  Same tolerances; within a few per cent of the default kernel either way.  Combined with
-     EI_FLAG_ATTN_PERSISTENT: one CTA per SM with a scheduler warp and a ring of item records; combined with
-     EI_FLAG_ATTN_SINGLE_TILE: one 128-row tile per CTA, two CTAs per SM.                                   */
-  EI_FLAG_ATTN_QUAD = 1u << 10
+  /* The quad-layout kernels (head_dim 128, block_len 128, segments a multiple of 256): sixteen softmax warps,
+     each owning sixteen query rows and all 128 key columns of a block through the 16-lane tensor-memory shapes,
+     so that the row maximum needs only two shuffles inside a quad of threads and no exchange between warps;
+     per-item records (list offset, visible and masked block counts) are worked out once per plan.  The form with
+     one CTA per tile pair is what ei_sparse_prefill runs on these shapes when no attention flag is given.  This
+     flag selects the other two forms: with EI_FLAG_ATTN_PERSISTENT one CTA per SM with a scheduler warp and a
+     ring of item records, with EI_FLAG_ATTN_SINGLE_TILE one 128-row tile per CTA and two CTAs per SM (both
+     bit-identical to the default and a few per cent slower in the measurements kept under profiles/).        */
+  EI_FLAG_ATTN_QUAD = 1u << 10,
+  /* Attention by the split-row kernel (same shapes; the default before the quad-layout kernel): two softmax threads
+     per query row in different warps, which agree on the row maximum through shared memory.  Within a few per
+     cent of the default; the only kernel that implements EI_FLAG_ATTN_SKIP_ZERO_PV (which implies it).      */
+  EI_FLAG_ATTN_SPLIT = 1u << 11
 } ei_flags;
 
 /* Fills *p with the paper's constants (e_t 1e-5, alpha 0.5, delta_t 0.4, cap 3, B_h 2048,
@@ -285,8 +290,8 @@ int ei_plan_status(ei_plan_t* plan, void* stream);
    every later wait returns at once, the kernels run to their common end, wait for their own copies in flight,
    free their tensor memory and return.  This call makes that path reachable without a faulty GPU:
    wait_limit_log2 > 0 shortens the bound of the plan's kernels to 2^wait_limit_log2 clocks (0: the default),
-   and skip_ring_item >= 0 makes the producer warp of the default stage-4 kernel (head_dim 128, block_len 128,
-   segments a multiple of 256) leave out that K/V load of every tile pair (item 2j is K of the j-th listed
+   and skip_ring_item >= 0 makes the producer warp of the default stage-4 kernel and of the split-row kernel
+   (head_dim 128, block_len 128, segments a multiple of 256) leave out that K/V load of every tile pair (item 2j is K of the j-th listed
    block, 2j + 1 its V; -1: none), so that the consumer's wait for it runs out.  ei_plan_status then reports
    the timeout and clears it; after ei_plan_debug_waits(plan, 0, -1, stream) the plan works as before.
    Host-synchronous on `stream`.  No counterpart in the paper.                                             */

@@ -24,6 +24,7 @@ from .binding import (  # noqa: F401
     FLAG_ATTN_NO_SKIP,
     FLAG_ATTN_SKIP_ZERO_PV,
     FLAG_ATTN_QUAD,
+    FLAG_ATTN_SPLIT,
     ROPE_NO_POOL,
     entropy_noalloc,
     lib,

@@ -358,6 +358,12 @@ int ei_stage_select(ei_plan_t* pl, void* stream) {
   if (e == cudaSuccess) {
     pl->planned = true;
     pl->items_valid = false;
+    // the per-item records of stage 4 follow from the lists alone: made here, once per plan
+    if (pl->shape.L_S % 256 == 0 && pl->shape.d == 128 && pl->shape.L_B == 128) {
+      e = ei::launch_attention_items(pl->lshape, pl->offsets, pl->indices, pl->items, (cudaStream_t)stream);
+      pl->launches += 1;
+      pl->items_valid = e == cudaSuccess;
+    }
   }
   return e == cudaSuccess ? EI_OK : EI_ERR_CUDA;
 }
@@ -442,9 +448,15 @@ static int attend(ei_plan_t* pl, const void* q, const void* k, const void* v, vo
   a.single_tile = (pl->params.flags & EI_FLAG_ATTN_SINGLE_TILE) != 0;
   a.pair_8warp = (pl->params.flags & EI_FLAG_ATTN_PAIR_8WARP) != 0;
   a.persistent = (pl->params.flags & EI_FLAG_ATTN_PERSISTENT) != 0;
-  a.quad_kernel = (pl->params.flags & EI_FLAG_ATTN_QUAD) != 0;
+  // head_dim 128, 128-wide blocks, segments a multiple of 256: the quad-layout kernel, one CTA per tile pair, unless
+  // a flag asks for another kernel (the split-row kernels are the only ones that can leave out all-zero P.V products)
+  const bool quad_shape = full.L_S % 256 == 0 && full.d == 128 && full.L_B == 128;
+  const uint32_t other = EI_FLAG_ATTN_SPLIT | EI_FLAG_ATTN_SKIP_ZERO_PV | EI_FLAG_ATTN_P_VIA_SMEM | EI_FLAG_ATTN_PAIR_8WARP;
+  a.quad_kernel = quad_shape && !(pl->params.flags & other) &&
+                  ((pl->params.flags & EI_FLAG_ATTN_QUAD) ||
+                   !(pl->params.flags & (EI_FLAG_ATTN_PERSISTENT | EI_FLAG_ATTN_SINGLE_TILE)));
   a.items = nullptr;
-  if (a.quad_kernel && full.L_S % 256 == 0) {
+  if (a.quad_kernel) {
     if (!pl->items_valid) {  // the lists changed since the records were made
       if (ei::launch_attention_items(pl->lshape, pl->offsets, pl->indices, pl->items, st) != cudaSuccess) return EI_ERR_CUDA;
       pl->items_valid = true;

@@ -28,6 +28,8 @@ Values are rounded once to bf16 (round-to-nearest-even); both sides read the sam
 """
 from __future__ import annotations
 
+import os
+from concurrent.futures import ThreadPoolExecutor
 from dataclasses import dataclass, replace
 
 import numpy as np
@@ -175,17 +177,30 @@ def gen_q_head(wl: Workload, st: Structure, h: int) -> np.ndarray:
     return f32_to_bf16_bits(q)
 
 
+def _workers() -> int:
+    return max(1, min(16, os.cpu_count() or 1))
+
+
 def generate(wl: Workload):
-    """-> (q [H,N,d], k [Hkv,N,d], v [Hkv,N,d]) uint16 bf16 bits, and the Structure."""
+    """-> (q [H,N,d], k [Hkv,N,d], v [Hkv,N,d]) uint16 bf16 bits, and the Structure.
+
+    Every head draws from a stream of its own, so the heads are generated by a pool of threads (numpy releases
+    the interpreter lock while it draws); the result does not depend on how many threads there are."""
     st = structure(wl)
     q = np.empty((wl.H, wl.N, wl.d), np.uint16)
     k = np.empty((wl.Hkv, wl.N, wl.d), np.uint16)
     v = np.empty((wl.Hkv, wl.N, wl.d), np.uint16)
-    for g in range(wl.Hkv):
+
+    def kv(g):
         k[g] = gen_k_head(wl, st, g)
         v[g] = gen_v_head(wl, g)
-    for h in range(wl.H):
+
+    def qh(h):
         q[h] = gen_q_head(wl, st, h)
+
+    with ThreadPoolExecutor(_workers()) as pool:
+        list(pool.map(kv, range(wl.Hkv)))
+        list(pool.map(qh, range(wl.H)))
     return q, k, v, st
 
 
@@ -193,9 +208,12 @@ def generate_plain(H: int, Hkv: int, N: int, d: int, seed: int, scale: float = 1
     """Structure-free N(0, scale^2) Q/K/V (bf16 bits) for exercising diffuse softmax rows."""
     def t(tensor, heads):
         out = np.empty((heads, N, d), np.uint16)
-        for h in range(heads):
+
+        def one(h):
             x = _rng(seed, tensor, h).standard_normal((N, d), dtype=np.float32)
             out[h] = f32_to_bf16_bits(x * np.float32(scale))
+        with ThreadPoolExecutor(_workers()) as pool:
+            list(pool.map(one, range(heads)))
         return out
     return t(_T_Q, H), t(_T_K, Hkv), t(_T_V, Hkv)
 

@@ -283,7 +283,8 @@ ATT_SHAPES = [
 
 @pytest.mark.parametrize("shape", ATT_SHAPES)
 @pytest.mark.parametrize("flags", [0, ei.FLAG_ATTN_P_VIA_SMEM, ei.FLAG_ATTN_SINGLE_TILE, ei.FLAG_ATTN_PAIR_8WARP,
-                                   ei.FLAG_ATTN_PERSISTENT, ei.FLAG_ATTN_PER_CTA, ei.FLAG_ATTN_QUAD,
+                                   ei.FLAG_ATTN_PERSISTENT, ei.FLAG_ATTN_PER_CTA, ei.FLAG_ATTN_SPLIT,
+                                   ei.FLAG_ATTN_SPLIT | ei.FLAG_ATTN_NO_SKIP,
                                    ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_NO_SKIP, ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_PERSISTENT,
                                    ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_PERSISTENT | ei.FLAG_ATTN_NO_SKIP,
                                    ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_SINGLE_TILE,
@@ -306,7 +307,7 @@ def test_attention_on_plain_inputs(shape, flags, lists):
 
 
 @pytest.mark.parametrize("flags", [0, ei.FLAG_ATTN_SINGLE_TILE, ei.FLAG_ATTN_PAIR_8WARP, ei.FLAG_ATTN_PERSISTENT,
-                                   ei.FLAG_ATTN_PER_CTA, ei.FLAG_ATTN_QUAD,
+                                   ei.FLAG_ATTN_PER_CTA, ei.FLAG_ATTN_SPLIT,
                                    ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_PERSISTENT, ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_SINGLE_TILE])
 @pytest.mark.parametrize("which", ["second_diag_only", "empty"])
 def test_attention_rows_without_visible_keys(flags, which):
@@ -455,7 +456,7 @@ def test_zero_p_products_left_out_is_bit_identical():
             q, k, v = synth.generate_plain(wl.H, wl.Hkv, wl.N, wl.d, seed=92)
         qd, kd, vd = to_dev(q), to_dev(k), to_dev(v)
         outs, left = [], []
-        for flags in (0, ei.FLAG_ATTN_SKIP_ZERO_PV, ei.FLAG_ATTN_SKIP_ZERO_PV | ei.FLAG_ATTN_NO_SKIP):
+        for flags in (ei.FLAG_ATTN_SPLIT, ei.FLAG_ATTN_SKIP_ZERO_PV, ei.FLAG_ATTN_SKIP_ZERO_PV | ei.FLAG_ATTN_NO_SKIP):
             pl = make_plan(wl, wl.fraction, flags=flags)
             pl.plan(qd, kd)
             out = torch.full((wl.H, wl.N, wl.d), float("nan"), dtype=torch.bfloat16, device="cuda")
@@ -536,7 +537,7 @@ def test_whole_path_edge_cases(name):
 
 
 @pytest.mark.parametrize("flags", [0, ei.FLAG_ATTN_SINGLE_TILE, ei.FLAG_ATTN_PAIR_8WARP, ei.FLAG_ATTN_PERSISTENT,
-                                   ei.FLAG_ATTN_PER_CTA, ei.FLAG_ATTN_QUAD,
+                                   ei.FLAG_ATTN_PER_CTA, ei.FLAG_ATTN_SPLIT,
                                    ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_PERSISTENT, ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_SINGLE_TILE])
 def test_attention_strided_tensors(flags):
     # q, k, v and out as views into wider buffers (token stride 3*d, as in a fused QKV activation)
@@ -655,26 +656,25 @@ def test_fused_and_staged_planning_agree_bit_for_bit(name):
 
 
 @pytest.mark.parametrize("name", ["mid128", "gqa7"])
-def test_persistent_attention_matches_the_per_cta_kernel_bit_for_bit(name):
-    # same arithmetic per tile, only the assignment of tiles to CTAs differs; two launches in a row also check
-    # that the item counter is back at zero after a launch
+def test_forms_of_a_kernel_family_agree_bit_for_bit(name):
+    # same arithmetic per tile, only the assignment of tiles to CTAs differs: the quad-layout kernels (one CTA per
+    # tile pair = the library's own choice, persistent, one tile per CTA) agree among themselves, and so do the two
+    # split-row kernels; two launches in a row also check that the item counter is back at zero after a launch
     wl = SMALL[name]
     q, k, v, st = synth.generate(wl)
     qd, kd, vd = to_dev(q), to_dev(k), to_dev(v)
-    outs = []
-    for flags in (ei.FLAG_ATTN_PER_CTA, ei.FLAG_ATTN_PERSISTENT, ei.FLAG_ATTN_PERSISTENT | ei.FLAG_GROUP_SHARED,
-                  ei.FLAG_GROUP_SHARED | ei.FLAG_ATTN_PER_CTA, 0):          # 0: the library's own choice
-        pl = make_plan(wl, wl.fraction, flags=flags)
-        pl.plan(qd, kd)
-        for rep in range(2):
-            out = torch.full((wl.H, wl.N, wl.d), float("nan"), dtype=torch.bfloat16, device="cuda")
-            pl.sparse_prefill(qd, kd, vd, out)
-            assert pl.status() == 0
-            outs.append(to_bits(out))
-    np.testing.assert_array_equal(outs[0], outs[1])
-    np.testing.assert_array_equal(outs[0], outs[2])
-    np.testing.assert_array_equal(outs[2], outs[3])
-    np.testing.assert_array_equal(outs[4], outs[6])
-    np.testing.assert_array_equal(outs[4], outs[5])
-    np.testing.assert_array_equal(outs[0], outs[8])
-    np.testing.assert_array_equal(outs[8], outs[9])
+    families = [(0, ei.FLAG_ATTN_PER_CTA, ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_PERSISTENT, ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_SINGLE_TILE),
+                (ei.FLAG_ATTN_SPLIT, ei.FLAG_ATTN_PERSISTENT)]
+    for family in families:
+        for group in (0, ei.FLAG_GROUP_SHARED):
+            outs = []
+            for flags in family:
+                pl = make_plan(wl, wl.fraction, flags=flags | group)
+                pl.plan(qd, kd)
+                for rep in range(2):
+                    out = torch.full((wl.H, wl.N, wl.d), float("nan"), dtype=torch.bfloat16, device="cuda")
+                    pl.sparse_prefill(qd, kd, vd, out)
+                    assert pl.status() == 0
+                    outs.append(to_bits(out))
+            for o in outs[1:]:
+                np.testing.assert_array_equal(outs[0], o)
