@@ -352,18 +352,13 @@ int ei_stage_budget(ei_plan_t* pl, void* stream) {
 int ei_stage_select(ei_plan_t* pl, void* stream) {
   if (!pl) return EI_ERR_INVALID_ARG;
   if (!on_plan_device(pl)) return EI_ERR_WRONG_DEVICE;
+  const bool quad_shape = pl->shape.L_S % 256 == 0 && pl->shape.d == 128 && pl->shape.L_B == 128;
   cudaError_t e = ei::launch_select(pl->lshape, pl->group ? pl->g_scores : pl->scores, pl->kblocks, pl->offsets,
-                                    pl->indices, (cudaStream_t)stream);
+                                    pl->indices, quad_shape ? pl->items : nullptr, (cudaStream_t)stream);
   pl->launches += 1;
   if (e == cudaSuccess) {
     pl->planned = true;
-    pl->items_valid = false;
-    // the per-item records of stage 4 follow from the lists alone: made here, once per plan
-    if (pl->shape.L_S % 256 == 0 && pl->shape.d == 128 && pl->shape.L_B == 128) {
-      e = ei::launch_attention_items(pl->lshape, pl->offsets, pl->indices, pl->items, (cudaStream_t)stream);
-      pl->launches += 1;
-      pl->items_valid = e == cudaSuccess;
-    }
+    pl->items_valid = quad_shape;  // the per-item records of stage 4 follow from the lists alone: made with them
   }
   return e == cudaSuccess ? EI_OK : EI_ERR_CUDA;
 }

@@ -1131,42 +1131,10 @@ __global__ void attention_items_kernel(const int* __restrict__ offsets, const in
   const long long rec = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (rec >= n_rec) return;
-  const int BN = s.L_B;
   const long long cell = rec / pairs_per_seg;
-  const int pr = (int)(rec % pairs_per_seg);
-  const int i = (int)(cell % s.C_S);
-  const long long q0 = (long long)i * s.L_S + (long long)pr * 2 * QBM;
-  int off = 0, n0 = 0, n1 = 0, jm0 = 0, jm1 = 0, blk0 = 0;
-  if (q0 < s.Nq) {  // a pair beyond the sequence (short last segment) keeps n0 = n1 = 0
-    off = __ldg(offsets + cell);
-    const int nlist = __ldg(offsets + cell + 1) - off;
-    // The list is ascending, so the blocks a tile does not see at all, and the blocks that need the causal mask,
-    // are suffixes of it: every lane looks at one entry from the tail, ballots count the suffixes.
-    int cut1 = 0, cut0 = 0, msk1 = 0, msk0 = 0;
-    for (int b0 = 0; b0 < nlist; b0 += 32) {
-      const int e = nlist - 1 - b0 - lane;
-      const bool in = e >= 0;
-      const long long blk = in ? (long long)__ldg(indices + off + e) : -1;
-      const unsigned c1 = __ballot_sync(0xffffffffu, in && blk * BN > q0 + s.P + 2 * QBM - 1);
-      const unsigned c0 = __ballot_sync(0xffffffffu, in && blk * BN > q0 + s.P + QBM - 1);
-      const unsigned m1 = __ballot_sync(0xffffffffu, in && (blk + 1) * BN - 1 > q0 + QBM + s.P);
-      const unsigned m0 = __ballot_sync(0xffffffffu, in && (blk + 1) * BN - 1 > q0 + s.P);
-      cut1 += __popc(c1);
-      cut0 += __popc(c0);
-      msk1 += __popc(m1);
-      msk0 += __popc(m0);
-      if (m0 != 0xffffffffu) break;  // the widest suffix ended inside this window
-    }
-    n1 = nlist - cut1;
-    n0 = nlist - cut0;
-    jm1 = nlist - msk1 < n1 ? nlist - msk1 : n1;
-    jm0 = nlist - msk0 < n0 ? nlist - msk0 : n0;
-    blk0 = nlist > 0 ? __ldg(indices + off) : 0;
-  }
-  if (lane < 8) {
-    const int v = lane == 0 ? off : lane == 1 ? n0 : lane == 2 ? n1 : lane == 3 ? jm0 : lane == 4 ? jm1 : lane == 5 ? blk0 : 0;
-    items[rec * 8 + lane] = v;
-  }
+  const int off = __ldg(offsets + cell);
+  attention_item_record(s, (int)(cell % s.C_S), (int)(rec % pairs_per_seg), off, __ldg(offsets + cell + 1) - off,
+                        indices + off, items + rec * 8, lane);
 }
 
 cudaError_t launch_attention_items(const Shape& ls, const int* offsets, const int* indices, int* items, cudaStream_t st) {

@@ -80,8 +80,9 @@ cudaError_t launch_budget(const Shape& s, const BudgetArgs& a, const float* entr
                           unsigned char* rigid, int* Mfx, int* kblocks, int* offsets, Stats* stats,
                           cudaStream_t st);
 
+// items (may be null): the stage-4 records of every (cell, tile pair), written by the warp that made the cell's list
 cudaError_t launch_select(const Shape& s, const float* scores, const int* kblocks,
-                          const int* offsets, int* indices, cudaStream_t st);
+                          const int* offsets, int* indices, int* items, cudaStream_t st);
 
 struct AttnArgs {
   const __nv_bfloat16 *q, *k, *v;
@@ -107,6 +108,46 @@ int launch_attention_quad(const Shape& s, const AttnArgs& a, cudaStream_t st);  
 // one record of 8 ints per (list cell, tile pair) from the plan's lists (ls: the list-head shape); a no-op for
 // shapes the tile-pair kernels do not take
 cudaError_t launch_attention_items(const Shape& ls, const int* offsets, const int* indices, int* items, cudaStream_t st);
+
+#ifdef __CUDACC__
+// Stage-4 record of one (list cell, tile pair): what a CTA has to know about its pair of 128-row query tiles before it
+// can start -- where the cell's ascending block list is, how many of its blocks each of the two tiles sees at all
+// (n0, n1), from which entry on they need the causal mask (jm0, jm1) and the first block.  Called by a whole warp
+// (`list` holds the cell's nlist entries; they may have been written by this warp just before, hence the L2
+// loads); lanes 0-7 store the record {off, n0, n1, jm0, jm1, blk0, 0, 0}.
+__device__ __forceinline__ void attention_item_record(const Shape& s, int seg, int pr, int off, int nlist,
+                                                      const int* list, int* rec, int lane) {
+  constexpr int TILE = 128;
+  const int BN = s.L_B;
+  const long long q0 = (long long)seg * s.L_S + (long long)pr * 2 * TILE;
+  int n0 = 0, n1 = 0, jm0 = 0, jm1 = 0, blk0 = 0;
+  if (q0 < s.Nq) {  // a pair beyond the sequence (short last segment) keeps n0 = n1 = 0
+    // The list is ascending, so the blocks a tile does not see at all, and the blocks that need the causal mask,
+    // are suffixes of it: every lane looks at one entry from the tail, ballots count the suffixes.
+    int cut1 = 0, cut0 = 0, msk1 = 0, msk0 = 0;
+    for (int b0 = 0; b0 < nlist; b0 += 32) {
+      const int e = nlist - 1 - b0 - lane;
+      const bool in = e >= 0;
+      const long long blk = in ? (long long)__ldcg(list + e) : -1;
+      const unsigned c1 = __ballot_sync(0xffffffffu, in && blk * BN > q0 + s.P + 2 * TILE - 1);
+      const unsigned c0 = __ballot_sync(0xffffffffu, in && blk * BN > q0 + s.P + TILE - 1);
+      const unsigned m1 = __ballot_sync(0xffffffffu, in && (blk + 1) * BN - 1 > q0 + TILE + s.P);
+      const unsigned m0 = __ballot_sync(0xffffffffu, in && (blk + 1) * BN - 1 > q0 + s.P);
+      cut1 += __popc(c1);
+      cut0 += __popc(c0);
+      msk1 += __popc(m1);
+      msk0 += __popc(m0);
+      if (m0 != 0xffffffffu) break;  // the widest suffix ended inside this window
+    }
+    n1 = nlist - cut1;
+    n0 = nlist - cut0;
+    jm1 = nlist - msk1 < n1 ? nlist - msk1 : n1;
+    jm0 = nlist - msk0 < n0 ? nlist - msk0 : n0;
+    blk0 = nlist > 0 ? __ldcg(list) : 0;
+  }
+  if (lane < 8) rec[lane] = lane == 0 ? off : lane == 1 ? n0 : lane == 2 ? n1 : lane == 3 ? jm0 : lane == 4 ? jm1 : lane == 5 ? blk0 : 0;
+}
+#endif
 
 // bf16 tensor [heads, N, d] (d contiguous) as a 3-D tensor map, box = 64 x box_rows x 1, 128-byte swizzle
 bool make_tensor_map(CUtensorMap* tm, const void* ptr, int d, int N, int heads, int64_t tok_stride,

@@ -907,76 +907,20 @@ budget_kernel(Shape s, BudgetArgs a, const float* __restrict__ entropy, unsigned
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return (long long)v;  // the same value in every thread
   };
-  // totals for NW candidates at once: every thread evaluates its cells at all of them, one block reduction per
-  // round (the same value in every thread afterwards)
-  constexpr int NW = 15;
-  __shared__ int s_multi[32][NW];
-  auto block_totals = [&](const long long (&cand)[NW], long long (&tot)[NW]) {
-    int t[NW];
-#pragma unroll
-    for (int w = 0; w < NW; ++w) {
-      const int bh = (int)(cand[w] >> 12), bl = (int)(cand[w] & 4095);
-      int acc = 0;
-      if (cpt <= CACHE) {
-#pragma unroll
-        for (int u = 0; u < CACHE; ++u)
-          if (c0 + u < c1) {
-            const int raw = (Mreg[u] * bh + ((Mreg[u] * bl) >> 12)) >> 12;
-            acc += min(max(raw, s.r), Creg[u]);
-          }
-      } else {
-        for (int c = c0, i = i_first; c < c1; ++c, i = (i + 1 == s.C_S ? 0 : i + 1)) {
-          const int M = Mfx[c];
-          const int raw = (M * bh + ((M * bl) >> 12)) >> 12;
-          acc += min(max(raw, s.r), causal_blocks(s, i));
-        }
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-      t[w] = acc;
-    }
-    __syncthreads();  // s_multi free again
-    if (lane == 0) {
-#pragma unroll
-      for (int w = 0; w < NW; ++w) s_multi[warp][w] = t[w];
-    }
-    __syncthreads();
-#pragma unroll
-    for (int w = 0; w < NW; ++w) {
-      int v = s_multi[lane][w];
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-      tot[w] = v;
-    }
-  };
   long long bstar;
   if (a.mode == EI_BUDGET_BASE_TOKENS) {
     bstar = a.b_fx_base;
   } else {
-    // the largest b with total(b) <= T: total is monotone in b, so any search finds the same b; sixteen-way
-    // instead of two-way cuts the block-wide rounds from 22 to 6
     long long lo = 0, hi = 4096LL * s.C_B;  // total(0) = cells*r <= T was checked on the host
     if (block_total(hi) <= a.T) {
       lo = hi;
     } else {
       while (hi - lo > 1) {  // invariant: total(lo) <= T < total(hi)
-        const long long step = (hi - lo + NW) / (NW + 1);  // >= 1
-        long long cand[NW], tot[NW];
-#pragma unroll
-        for (int w = 0; w < NW; ++w) {
-          const long long c = lo + (w + 1) * step;
-          cand[w] = c < hi ? c : hi;  // (a candidate equal to hi is known to exceed T; it keeps the arrays full)
-        }
-        block_totals(cand, tot);
-        long long nlo = lo, nhi = hi;
-#pragma unroll
-        for (int w = 0; w < NW; ++w) {
-          if (cand[w] < hi && tot[w] <= a.T) nlo = cand[w];
-          else if (cand[w] < nhi && cand[w] > nlo && (cand[w] >= hi || tot[w] > a.T)) nhi = cand[w] < nhi ? cand[w] : nhi;
-        }
-        // candidates ascend and total is monotone: nlo is the last one within T, nhi the first one beyond it
-        lo = nlo;
-        hi = nhi;
+        const long long mid = lo + (hi - lo) / 2;
+        if (block_total(mid) <= a.T)
+          lo = mid;
+        else
+          hi = mid;
       }
     }
     bstar = lo;
@@ -1057,7 +1001,7 @@ __device__ __forceinline__ uint32_t order_key(float f) {
 
 __global__ void __launch_bounds__(SEL_WARPS * 32)
 select_kernel(Shape s, const float* __restrict__ scores, const int* __restrict__ kblocks,
-              const int* __restrict__ offsets, int* __restrict__ indices) {
+              const int* __restrict__ offsets, int* __restrict__ indices, int* __restrict__ items, int pairs_per_seg) {
   __shared__ int hist[SEL_WARPS][256];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const long long c = (long long)blockIdx.x * SEL_WARPS + warp;
@@ -1143,12 +1087,18 @@ select_kernel(Shape s, const float* __restrict__ scores, const int* __restrict__
     }
   }
   for (int t = lane; t < nd && t < k; t += 32) out[written + t] = ncand + t;
+  if (items != nullptr) {  // the list is complete: the stage-4 records of this cell's tile pairs follow from it
+    __syncwarp();
+    for (int pr = 0; pr < pairs_per_seg; ++pr)
+      attention_item_record(s, i, pr, offsets[c], k, out, items + (c * pairs_per_seg + pr) * 8, lane);
+  }
 }
 
 cudaError_t launch_select(const Shape& s, const float* scores, const int* kblocks, const int* offsets,
-                          int* indices, cudaStream_t st) {
+                          int* indices, int* items, cudaStream_t st) {
   const unsigned grid = (unsigned)((s.cells + SEL_WARPS - 1) / SEL_WARPS);
-  select_kernel<<<grid, SEL_WARPS * 32, 0, st>>>(s, scores, kblocks, offsets, indices);
+  const int pairs = s.L_S % 256 == 0 ? s.L_S / 256 : 0;  // shapes the tile-pair kernels of stage 4 take
+  select_kernel<<<grid, SEL_WARPS * 32, 0, st>>>(s, scores, kblocks, offsets, indices, pairs ? items : nullptr, pairs);
   return cudaGetLastError();
 }
 
