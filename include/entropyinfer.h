@@ -70,7 +70,17 @@ typedef struct ei_params {
   uint32_t struct_size;        /* sizeof(ei_params), for versioning                            */
   int32_t n_q_heads;           /* H                                                            */
   int32_t n_kv_heads;          /* H_kv; query head h reads KV head h / (H / H_kv)              */
-  int32_t head_dim;            /* d: 64, 128 or 256 (256: planning in two passes over d, one-tile attention kernel) */
+  int32_t head_dim;            /* d: 64, 128 or 256 (256: planning in two passes over d, one-tile attention kernel).
+                                  Other widths (96, 192) return EI_ERR_UNSUPPORTED_SHAPE, by design: a row of
+                                  Q / K is streamed as a power-of-two number of 16-byte lanes (pooling gives each
+                                  lane one thread of a power-of-two team and reduces the team by shuffles), the
+                                  fp64 observation kernel stages d in 64-wide passes of a fixed count, and the
+                                  attention kernels lay the operands out as whole pairs of 64-column swizzled
+                                  panels with O in a power-of-two tensor-memory allocation (a 192-wide O next to
+                                  S leaves no room for the second tile).  Pad such heads to the next supported
+                                  width with zero columns: logits, entropies, selections and outputs are
+                                  unchanged (the added output columns are zero) when obs_scale and attn_scale are
+                                  given as 1/sqrt(true d).                                                    */
   int32_t seq_len;             /* N; need not be a multiple of segment_len or block_len: there are then
                                   C_S = ceil(N/L_S) segments and C_B = ceil(N/L_B) key blocks, the short
                                   last segment / block is pooled over the rows it has, segment i sees

@@ -555,6 +555,32 @@ def test_ragged_total_mode_and_full_budget_attention():
         assert 12 in p2.idx[p2.offsets[cc]:p2.offsets[cc + 1]].tolist()
 
 
+def test_short_last_segment_keeps_r_blocks_not_its_diagonal_count():
+    # N = 400 with L_S = 64, L_B = 32 (r = 2): 13 key blocks; the last segment (rows 384..399) has ONE diagonal
+    # block (12) and sees all 13.  With the base budget far below one block every cell is forced to its minimum,
+    # and that minimum is r = 2 for every segment that sees at least r blocks -- the unchanged formula
+    # k = min(C_i, max(r, .)) -- not the segment's diagonal count (which would give 1 here).  Worked by hand:
+    #   k = [2, 2, 2, 2, 2, 2, 2];  the last list = {12} (forced) + the best of blocks 0..11.
+    m = np.ones((1, 7), np.float64)
+    k = oracle.budgets_base(m, 2, 0.01, C_B=13)
+    np.testing.assert_array_equal(k[0], [2, 2, 2, 2, 2, 2, 2])
+    # TOTAL mode at the smallest feasible total: sum of min(r, C_i) = 14, again 2 in the short segment;
+    # one block fewer is infeasible (the diagonal-count reading would accept 13)
+    kt, _ = oracle.budgets_total(m, 2, 14, C_B=13)
+    np.testing.assert_array_equal(kt[0], [2, 2, 2, 2, 2, 2, 2])
+    with pytest.raises(ValueError):
+        oracle.budgets_total(m, 2, 13, C_B=13)
+    # selection: the short segment's list is its diagonal block plus the highest-scoring other block (block 5 here)
+    lnA = np.full((1, 55), -9.0, np.float64)
+    last = oracle.row_offset(6, 2)
+    lnA[0, last + 5] = -1.0
+    lnA[0, last + 12] = -20.0                      # the diagonal block is kept however low it scores
+    off, idx, _ = oracle.select(lnA, k, 2, C_B=13)
+    assert sorted(idx[off[6]:off[7]].tolist()) == [5, 12]
+    # a sequence shorter than one segment with a single block: C_i = 1 < r, the cap wins
+    np.testing.assert_array_equal(oracle.budgets_base(np.ones((1, 1)), 2, 0.01, C_B=1), [[1]])
+
+
 # ---------------------------------------------------------------- chunked prefill: the queries are a suffix of the keys
 def test_chunked_counts_by_hand():
     # N = 512 keys in 16 blocks of 32, the last 160 positions are the queries: c0 = 11 blocks lie before them,
