@@ -36,7 +36,7 @@ NCU_COUNTERS = os.path.join(ROOT, "profiles", "ncu_counters_attention.txt")
 KERNEL_SOURCES = {"sparse_attention_quad_kernel": "ei_attention_quad.cu", "sparse_attention_quad_persistent_kernel": "ei_attention_quad.cu",
                   "sparse_attention_quad1_kernel": "ei_attention_quad.cu", "sparse_attention_split_kernel": "ei_attention.cu",
                   "sparse_attention_persistent_kernel": "ei_attention.cu", "sparse_attention_pair_kernel": "ei_attention.cu",
-                  "sparse_attention_kernel": "ei_attention.cu"}
+                  "sparse_attention_kernel": "ei_attention.cu", "sparse_attention_tri_kernel": "ei_attention_tri.cu"}
 
 
 def git_blob_hash(path: str) -> str:
@@ -596,13 +596,13 @@ def run_ours(args, wl):
 ATTENTION_CHOICES = {"default": "sparse_attention_quad_kernel", "per_cta": "sparse_attention_quad_kernel",
                      "quad_persistent": "sparse_attention_quad_persistent_kernel",
                      "quad_single_tile": "sparse_attention_quad1_kernel", "split": "sparse_attention_split_kernel",
-                     "persistent": "sparse_attention_persistent_kernel"}
+                     "persistent": "sparse_attention_persistent_kernel", "tri": "sparse_attention_tri_kernel"}
 
 
 def attention_flags(ei, choice: str) -> int:
     return {"default": 0, "per_cta": ei.FLAG_ATTN_PER_CTA, "quad_persistent": ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_PERSISTENT,
             "quad_single_tile": ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_SINGLE_TILE, "split": ei.FLAG_ATTN_SPLIT,
-            "persistent": ei.FLAG_ATTN_PERSISTENT}[choice]
+            "persistent": ei.FLAG_ATTN_PERSISTENT, "tri": ei.FLAG_ATTN_TRI}[choice]
 
 
 def attention_kernel_name(wl, args, total_blocks) -> str:
@@ -732,7 +732,7 @@ def main():
                     help="also time the rotary producer with and without the pooling folded in (ei_rope_pool, ei_plan_pooled)")
     ap.add_argument("--with-compress", action="store_true", help="also time the Alg. 4 KV-cache compression")
     ap.add_argument("--attention", default="default", choices=sorted(ATTENTION_CHOICES),
-                    help="persistent: the persistent form of the two-threads-per-row attention kernel")
+                    help="persistent: the persistent form of the two-threads-per-row attention kernel; tri: the three-buffer kernel")
     ap.add_argument("--no-skip", action="store_true",
                     help="evaluate every probability (EI_FLAG_ATTN_NO_SKIP): no shortcut for negligible half rows")
     ap.add_argument("--graph", action="store_true", help="also time the step replayed from a CUDA graph")

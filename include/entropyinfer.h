@@ -165,7 +165,12 @@ typedef enum ei_flags {
   /* Attention by the split-row kernel (same shapes; the default before the quad-layout kernel): two softmax threads
      per query row in different warps, which agree on the row maximum through shared memory.  Within a few per
      cent of the default; the only kernel that implements EI_FLAG_ATTN_SKIP_ZERO_PV (which implies it).      */
-  EI_FLAG_ATTN_SPLIT = 1u << 11
+  EI_FLAG_ATTN_SPLIT = 1u << 11,
+  /* Attention by the three-buffer kernel (same shapes): one 128-row tile at a time per CTA with three S buffers
+     and one O in tensor memory, Q.K^T three key blocks ahead of P.V, two sets of softmax warps on alternate key
+     blocks that pass the row reference maxima to each other through shared memory; a CTA runs through several
+     consecutive tiles of a segment.                                                                          */
+  EI_FLAG_ATTN_TRI = 1u << 12
 } ei_flags;
 
 /* Fills *p with the paper's constants (e_t 1e-5, alpha 0.5, delta_t 0.4, cap 3, B_h 2048,

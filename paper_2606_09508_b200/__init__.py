@@ -25,6 +25,7 @@ from .binding import (  # noqa: F401
     FLAG_ATTN_SKIP_ZERO_PV,
     FLAG_ATTN_QUAD,
     FLAG_ATTN_SPLIT,
+    FLAG_ATTN_TRI,
     ROPE_NO_POOL,
     entropy_noalloc,
     lib,

@@ -56,6 +56,7 @@ FLAG_ATTN_NO_SKIP = 256
 FLAG_ATTN_SKIP_ZERO_PV = 512
 FLAG_ATTN_QUAD = 1024
 FLAG_ATTN_SPLIT = 2048
+FLAG_ATTN_TRI = 4096
 
 # every symbol the header declares: (name, restype, argtypes)
 _P = C.c_void_p

@@ -6,7 +6,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libentropyinfer.so")
-SOURCES = ["ei_api.cu", "ei_plan_kernels.cu", "ei_attention.cu", "ei_attention_quad.cu", "ei_noalloc.cu", "ei_compress.cu", "ei_producer.cu"]
+SOURCES = ["ei_api.cu", "ei_plan_kernels.cu", "ei_attention.cu", "ei_attention_quad.cu", "ei_attention_tri.cu", "ei_noalloc.cu", "ei_compress.cu", "ei_producer.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I" + INCLUDE, "-I" + CSRC]
 

@@ -450,8 +450,11 @@ static int attend(ei_plan_t* pl, const void* q, const void* k, const void* v, vo
   a.quad_kernel = quad_shape && !(pl->params.flags & other) &&
                   ((pl->params.flags & EI_FLAG_ATTN_QUAD) ||
                    !(pl->params.flags & (EI_FLAG_ATTN_PERSISTENT | EI_FLAG_ATTN_SINGLE_TILE)));
+  a.tri_kernel = quad_shape && (pl->params.flags & EI_FLAG_ATTN_TRI) != 0;
+  a.tri_tiles = 0;
+  if (a.tri_kernel) a.quad_kernel = false;
   a.items = nullptr;
-  if (a.quad_kernel) {
+  if (a.quad_kernel || a.tri_kernel) {
     if (!pl->items_valid) {  // the lists changed since the records were made
       if (ei::launch_attention_items(pl->lshape, pl->offsets, pl->indices, pl->items, st) != cudaSuccess) return EI_ERR_CUDA;
       pl->items_valid = true;

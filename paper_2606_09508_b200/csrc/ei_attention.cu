@@ -1754,6 +1754,7 @@ int launch_attention(const Shape& s, const AttnArgs& a, cudaStream_t st) {
     if (s.L_B == 64) return launch_t<256, 64, 2, false>(s, a, st);
     return EI_ERR_UNSUPPORTED_SHAPE;
   }
+  if (a.tri_kernel && s.L_S % (2 * BM) == 0 && s.d == 128 && s.L_B == 128) return launch_attention_tri(s, a, st);
   if (a.quad_kernel && s.L_S % (2 * BM) == 0 && s.d == 128 && s.L_B == 128) return launch_attention_quad(s, a, st);
   if (a.persistent && a.sched && s.L_S % (2 * BM) == 0 && s.d == 128 && s.L_B == 128)
     return launch_persistent_t<128, 128, 5>(s, a, st);

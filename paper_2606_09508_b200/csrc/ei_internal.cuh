@@ -96,6 +96,8 @@ struct AttnArgs {
   bool pair_8warp;   // force the two-tile kernel with one softmax thread per row
   bool persistent;   // the persistent form of the split-row kernel (items off a counter)
   bool quad_kernel;  // the quad-layout kernel (ei_attention_quad.cu)
+  bool tri_kernel;   // the three-buffer kernel (ei_attention_tri.cu); needs items like the quad-layout kernels
+  int tri_tiles;     // tiles per CTA of the three-buffer kernel (0: its default)
   int* sched;        // two ints, zero between launches: next item, CTAs finished
   float skip_log2;   // split-row kernels: half rows more than this many binary orders below the row maximum get P = 0
                      // without being exponentiated (infinity: never)
@@ -105,6 +107,7 @@ struct AttnArgs {
 // returns EI_OK or a negative ei_status (tensor-map encoding can fail)
 int launch_attention(const Shape& s, const AttnArgs& a, cudaStream_t st);
 int launch_attention_quad(const Shape& s, const AttnArgs& a, cudaStream_t st);  // d = 128, L_B = 128, L_S % 256 = 0
+int launch_attention_tri(const Shape& s, const AttnArgs& a, cudaStream_t st);   // same shapes
 // one record of 8 ints per (list cell, tile pair) from the plan's lists (ls: the list-head shape); a no-op for
 // shapes the tile-pair kernels do not take
 cudaError_t launch_attention_items(const Shape& ls, const int* offsets, const int* indices, int* items, cudaStream_t st);

@@ -155,6 +155,54 @@ __device__ __forceinline__ void umma_ts(uint32_t d, uint32_t a, uint64_t bdesc, 
       ::"r"(d), "r"(a), "l"(bdesc), "r"(idesc), "r"(accum)
       : "memory");
 }
+// Eight K = 16 steps of S = Q . K^T in one go (both operands in 128-byte-swizzled K-major tiles of two 64-column
+// panels 16 KB apart): one elected thread, one predicate set-up, the descriptors advanced by adds on their
+// 16-byte address field (+2 inside a panel, +1018 from the end of panel 0 to the start of panel 1).  Issuing
+// them one by one with a descriptor built per instruction costs the issuing warp more than the tensor pipe needs
+// to execute them.
+__device__ __forceinline__ void umma_ss_d128(uint32_t d, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
+  if (elect_one())
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 a, b;\n\t"
+        "mov.b64 a, %1;\n\tmov.b64 b, %2;\n\t"
+        "setp.ne.b32 p, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p;\n\t"
+        "setp.eq.b32 p, 0, 0;\n\t"
+        "add.s64 a, a, 2;\n\tadd.s64 b, b, 2;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p;\n\t"
+        "add.s64 a, a, 2;\n\tadd.s64 b, b, 2;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p;\n\t"
+        "add.s64 a, a, 2;\n\tadd.s64 b, b, 2;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p;\n\t"
+        "add.s64 a, a, 1018;\n\tadd.s64 b, b, 1018;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p;\n\t"
+        "add.s64 a, a, 2;\n\tadd.s64 b, b, 2;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p;\n\t"
+        "add.s64 a, a, 2;\n\tadd.s64 b, b, 2;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p;\n\t"
+        "add.s64 a, a, 2;\n\tadd.s64 b, b, 2;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p;\n\t}"
+        ::"r"(d), "l"(adesc), "l"(bdesc), "r"(idesc)
+        : "memory");
+}
+// Four K = 16 steps of O (+)= P . V (P from tensor memory, 8 packed columns per step; V MN-major, 2 KB per step)
+__device__ __forceinline__ void umma_ts_x4(uint32_t d, uint32_t a, uint64_t bdesc, uint32_t idesc, uint32_t accum_first) {
+  if (elect_one())
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 b;\n\t.reg .b32 a;\n\t"
+        "mov.b64 b, %2;\n\tmov.b32 a, %1;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, p;\n\t"
+        "setp.eq.b32 p, 0, 0;\n\t"
+        "add.s64 b, b, 128;\n\tadd.u32 a, a, 8;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, p;\n\t"
+        "add.s64 b, b, 128;\n\tadd.u32 a, a, 8;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, p;\n\t"
+        "add.s64 b, b, 128;\n\tadd.u32 a, a, 8;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, p;\n\t}"
+        ::"r"(d), "r"(a), "l"(bdesc), "r"(idesc), "r"(accum_first)
+        : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   if (elect_one())
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");

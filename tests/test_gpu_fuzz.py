@@ -21,6 +21,8 @@ def draw(seed):
         d = 256
     L_B = int(rng.choice([64, 128]))
     L_S = int(rng.choice([m for m in (128, 256, 512) if m % L_B == 0]))
+    if seed >= 200:                                              # a third family: the shape of the tile-pair kernels
+        d, L_B, L_S = 128, 128, (256, 512)[seed % 2]
     Hkv = int(rng.choice([1, 2, 3]))
     G = int(rng.choice([1, 2, 4, 7]))
     n_blocks = int(rng.integers(3, 40))
@@ -36,10 +38,12 @@ def draw(seed):
     flags |= int(rng.choice([0, ei.FLAG_ATTN_PERSISTENT, ei.FLAG_ATTN_SINGLE_TILE, ei.FLAG_ATTN_PAIR_8WARP, ei.FLAG_ATTN_PER_CTA]))
     if seed % 5 == 3:                                            # every fifth configuration: all probabilities evaluated
         flags |= ei.FLAG_ATTN_NO_SKIP
+    if seed >= 200:                                              # the three-buffer kernel where the shape allows it
+        flags |= ei.FLAG_ATTN_TRI
     return dict(H=Hkv * G, Hkv=Hkv, d=d, N=N, P=P, L_S=L_S, L_B=L_B, mode=mode, f=f, flags=flags, seed=seed)
 
 
-@pytest.mark.parametrize("seed", list(range(28)) + list(range(100, 112)))
+@pytest.mark.parametrize("seed", list(range(28)) + list(range(100, 112)) + list(range(200, 212)))
 def test_random_configuration(seed):
     c = draw(seed)
     H, Hkv, d, N, P, L_S, L_B = (c[k] for k in ("H", "Hkv", "d", "N", "P", "L_S", "L_B"))

@@ -288,7 +288,8 @@ ATT_SHAPES = [
                                    ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_NO_SKIP, ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_PERSISTENT,
                                    ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_PERSISTENT | ei.FLAG_ATTN_NO_SKIP,
                                    ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_SINGLE_TILE,
-                                   ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_SINGLE_TILE | ei.FLAG_ATTN_NO_SKIP])
+                                   ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_SINGLE_TILE | ei.FLAG_ATTN_NO_SKIP,
+                                   ei.FLAG_ATTN_TRI, ei.FLAG_ATTN_TRI | ei.FLAG_ATTN_NO_SKIP])
 @pytest.mark.parametrize("lists", ["full", "random", "diag"])
 def test_attention_on_plain_inputs(shape, flags, lists):
     # structure-free N(0,1) inputs: diffuse softmax rows in every head, every diagonal-mask case
@@ -308,7 +309,8 @@ def test_attention_on_plain_inputs(shape, flags, lists):
 
 @pytest.mark.parametrize("flags", [0, ei.FLAG_ATTN_SINGLE_TILE, ei.FLAG_ATTN_PAIR_8WARP, ei.FLAG_ATTN_PERSISTENT,
                                    ei.FLAG_ATTN_PER_CTA, ei.FLAG_ATTN_SPLIT,
-                                   ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_PERSISTENT, ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_SINGLE_TILE])
+                                   ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_PERSISTENT, ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_SINGLE_TILE,
+                                   ei.FLAG_ATTN_TRI])
 @pytest.mark.parametrize("which", ["second_diag_only", "empty"])
 def test_attention_rows_without_visible_keys(flags, which):
     # hand-made lists in which some (or all) 128-row tiles see no key at all: those rows must come
@@ -538,7 +540,8 @@ def test_whole_path_edge_cases(name):
 
 @pytest.mark.parametrize("flags", [0, ei.FLAG_ATTN_SINGLE_TILE, ei.FLAG_ATTN_PAIR_8WARP, ei.FLAG_ATTN_PERSISTENT,
                                    ei.FLAG_ATTN_PER_CTA, ei.FLAG_ATTN_SPLIT,
-                                   ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_PERSISTENT, ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_SINGLE_TILE])
+                                   ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_PERSISTENT, ei.FLAG_ATTN_QUAD | ei.FLAG_ATTN_SINGLE_TILE,
+                                   ei.FLAG_ATTN_TRI])
 def test_attention_strided_tensors(flags):
     # q, k, v and out as views into wider buffers (token stride 3*d, as in a fused QKV activation)
     H, Hkv, d, N, L_S, L_B = 4, 2, 128, 1024, 256, 128
