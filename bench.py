@@ -593,6 +593,209 @@ def run_ours(args, wl):
 # Parameter sweeps (speed only; the paper sweeps segment / block size and budgets for quality, Fig. 5-6, and
 # reports end-to-end latency against input length, Section 5.3).  One JSON line per point.
 # ----------------------------------------------------------------------------------------------
+# ----------------------------------------------------------------------------------------------
+# One layer's heads sharded over the ranks by KV group (--shard kv): strong scaling of ONE layer
+# ----------------------------------------------------------------------------------------------
+def shard_heads(H: int, Hkv: int, rank: int, world: int):
+    """Rank p of `world` holds the KV heads [p*Hkv/world, (p+1)*Hkv/world) and the query heads that read them."""
+    if Hkv % world != 0:
+        raise ValueError(f"{Hkv} KV heads do not split over {world} ranks")
+    g_per, G = Hkv // world, H // Hkv
+    g0 = rank * g_per
+    return g0 * G, (g0 + g_per) * G, g0, g0 + g_per
+
+
+def total_blocks_all(wl) -> int:
+    """T of the whole layer, as ei_plan_create works it out for a plan over all heads."""
+    SC = sum(min(wl.r * (i + 1), wl.C_B) for i in range(wl.C_S))
+    return int(math.floor(wl.fraction * float(wl.H) * float(SC) + 0.5))
+
+
+def run_shard_kv(args, wl):
+    """The layer of the workload with its heads sharded over the ranks by KV group.  Everything of the method is
+    per head except TOTAL mode's common total: every rank works out the multipliers of its heads, the int32
+    tables are all-gathered (NCCL, the one collective of the path), and every rank apportions the layer's total
+    over the gathered table and keeps its own rows.  Each rank then selects and attends for its heads alone."""
+    import torch
+
+    import paper_2606_09508_b200 as ei
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    peaks = load_peaks()
+    h0, h1, g0, g1 = shard_heads(wl.H, wl.Hkv, rank, world)
+    q, k, v, st = synth.generate(wl)          # every rank draws the layer (seeded), keeps its heads
+
+    def dev(b):
+        return torch.from_numpy(np.ascontiguousarray(b).view(np.int16)).cuda().view(torch.bfloat16)
+
+    qd, kd, vd = dev(q[h0:h1]), dev(k[g0:g1]), dev(v[g0:g1])
+    Hl, Hkvl = h1 - h0, g1 - g0
+    out = torch.empty((Hl, wl.N, wl.d), dtype=torch.bfloat16, device="cuda")
+    params = ei.params_default(Hl, Hkvl, wl.d, wl.N, wl.L_S, wl.L_B, wl.fraction)
+    params.flags |= ei.FLAG_HEAD_SHARD | attention_flags(ei, args.attention)
+    if args.no_skip:
+        params.flags |= ei.FLAG_ATTN_NO_SKIP
+    plan = ei.Plan(params)
+    stream = torch.cuda.current_stream()
+    T_all = total_blocks_all(wl)
+    m_all = torch.zeros((wl.H, wl.C_S), dtype=torch.int32, device="cuda")
+    m_loc = torch.zeros((Hl, wl.C_S), dtype=torch.int32, device="cuda")
+
+    def plan_step():
+        plan.observe(qd, kd)
+        if world > 1:
+            plan.stage_multipliers(out=m_loc)
+            dist.all_gather_into_tensor(m_all.view(-1), m_loc.view(-1))
+        else:
+            plan.stage_multipliers(out=m_all)
+        plan.stage_apportion(m_all, wl.H, h0, T_all)
+        plan.stage_select()
+
+    def step():
+        plan_step()
+        plan.sparse_prefill(qd, kd, vd, out)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    if plan.status() != 0:
+        raise RuntimeError("device-side wait timed out during warm-up")
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    launches0 = plan.launches()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_wall0 = time.time()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step()
+    ev1.record(stream)
+    barrier()
+    t_wall1 = time.time()
+    launches = plan.launches() - launches0
+    elapsed_ms = max_over_ranks(ev0.elapsed_time(ev1), dist, "cuda")
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    if plan.status() != 0:
+        raise RuntimeError("device-side wait timed out during the timed region")
+    ms_per_step = elapsed_ms / args.steps
+
+    # per-call timing on this rank (max over ranks): the planning sequence with its all-gather, the attention launch
+    pe = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    for s_ in range(args.steps):
+        pe[s_][0].record(stream)
+        plan_step()
+        pe[s_][1].record(stream)
+        plan.sparse_prefill(qd, kd, vd, out)
+        pe[s_][2].record(stream)
+    torch.cuda.synchronize()
+    plan_ms = max_over_ranks(float(np.mean([pe[s_][0].elapsed_time(pe[s_][1]) for s_ in range(args.steps)])), dist, "cuda")
+    attn_ms = max_over_ranks(float(np.mean([pe[s_][1].elapsed_time(pe[s_][2]) for s_ in range(args.steps)])), dist, "cuda")
+    res = plan.results()
+    tiles_local = executed_tiles(synth.generator.with_(wl, H=Hl, Hkv=Hkvl), res["k"])
+    tiles_t = torch.tensor([float(tiles_local)], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(tiles_t)
+    flops = float(tiles_t.item()) * tile_flops(wl)
+
+    # the shards against one plan over all heads (rank 0, which has drawn the whole layer): same rows, bit for bit
+    matches = None
+    if rank == 0 and not args.no_dense:
+        pf = ei.params_default(wl.H, wl.Hkv, wl.d, wl.N, wl.L_S, wl.L_B, wl.fraction)
+        pf.flags = params.flags & ~ei.FLAG_HEAD_SHARD
+        full = ei.Plan(pf)
+        qf, kf = dev(q), dev(k)
+        full.plan(qf, kf)
+        rf = full.results()
+        cells = Hl * wl.C_S
+        lo = int(rf["offsets"][h0 * wl.C_S])
+        matches = bool(np.array_equal(rf["k"][h0:h1], res["k"]) and
+                       np.array_equal(rf["offsets"][h0 * wl.C_S:h0 * wl.C_S + cells + 1] - lo, res["offsets"]) and
+                       np.array_equal(rf["idx"][lo:lo + int(res["offsets"][-1])], res["idx"][:int(res["offsets"][-1])]))
+        del full, qf, kf
+
+    # end to end: this rank's heads from pinned host buffers, result back to the host, every step
+    e2e = None
+    if not args.no_e2e:
+        hq, hk, hv = (torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).pin_memory()
+                      for a in (q[h0:h1], k[g0:g1], v[g0:g1]))
+        hout = torch.empty((Hl, wl.N, wl.d), dtype=torch.int16).pin_memory()
+        qi, ki, vi = (torch.empty_like(t_, device="cuda") for t_ in (hq, hk, hv))
+
+        def e2e_step():
+            qi.copy_(hq, non_blocking=True)
+            ki.copy_(hk, non_blocking=True)
+            vi.copy_(hv, non_blocking=True)
+            qb, kb, vb = (t_.view(torch.bfloat16) for t_ in (qi, ki, vi))
+            plan.observe(qb, kb)
+            if world > 1:
+                plan.stage_multipliers(out=m_loc)
+                dist.all_gather_into_tensor(m_all.view(-1), m_loc.view(-1))
+            else:
+                plan.stage_multipliers(out=m_all)
+            plan.stage_apportion(m_all, wl.H, h0, T_all)
+            plan.stage_select()
+            plan.sparse_prefill(qb, kb, vb, out)
+            hout.copy_(out.view(torch.int16), non_blocking=True)
+        e2e_step()
+        barrier()
+        n_e = max(2, min(args.steps, 5))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(n_e):
+            e2e_step()
+        e1.record(stream)
+        barrier()
+        e_ms = max_over_ranks(e0.elapsed_time(e1), dist, "cuda") / n_e
+        e2e = {"value": e_ms, "unit": "ms/layer", "h2d_bytes_per_step": int((hq.numel() + hk.numel() + hv.numel()) * 2),
+               "d2h_bytes_per_step": int(hout.numel() * 2), "steps": n_e,
+               "what": "per rank: its heads' Q, K, V up from pinned host memory, sharded planning, attention, output down"}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+    timed_s = ms_per_step * args.steps * 1e-3
+    peak_key = "bf16_tflops" if timed_s < 1.0 else "bf16_tflops_sustained"
+    att_tflops = flops / (attn_ms * 1e-3) / 1e12
+    kern = attention_kernel_name(wl, args, 0)
+    ctr = {"tensor_pipe_active_pct_ncu": None, "traffic": None, "stale": None}   # no capture of the sharded launch
+    cfg = workload_config(wl)
+    cfg["parallelism"] = f"one layer, heads sharded by KV group over {world} GPU(s): {Hkvl} KV heads + {Hl} query heads per rank"
+    cfg["exchange"] = "one all-gather of the int32 multiplier table (H x C_S) per step (NCCL)" if world > 1 else "none (one rank)"
+    line = {"metric": "128k-token sparse prefill attention ms/layer; tensor-pipe % of B200 peak", "value": ms_per_step,
+            "unit": "ms/layer", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "strong", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic", "config": cfg,
+            "kernel_ms": {"plan_with_exchange": plan_ms, "attention": attn_ms},
+            "executed_tflop": flops / 1e12,
+            "roofline": {"bound": "tensor", "achieved": att_tflops, "peak": peaks[peak_key] * world, "unit": "TFLOP/s",
+                         "frac": att_tflops / (peaks[peak_key] * world), "traffic": ctr["traffic"],
+                         "kernel": kern, "tensor_pipe_active_pct_ncu": ctr["tensor_pipe_active_pct_ncu"], "stale": ctr["stale"],
+                         "peak_kind": f"{world} x cuBLAS bf16 " + ("burst" if peak_key == "bf16_tflops" else "sustained") + " (measured)",
+                         "what": "all ranks' executed tiles / the slowest rank's attention launch"},
+            "shards_match_unsharded_plan": matches, "cpu_baseline": None, "e2e": e2e, "gpu_launches": int(launches),
+            "clocks": clocks}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+
 ATTENTION_CHOICES = {"default": "sparse_attention_quad_kernel", "per_cta": "sparse_attention_quad_kernel",
                      "quad_persistent": "sparse_attention_quad_persistent_kernel",
                      "quad_single_tile": "sparse_attention_quad1_kernel", "split": "sparse_attention_split_kernel",
@@ -738,6 +941,9 @@ def main():
     ap.add_argument("--graph", action="store_true", help="also time the step replayed from a CUDA graph")
     ap.add_argument("--group-shared", action="store_true",
                     help="plan once per KV group (EI_FLAG_GROUP_SHARED) instead of once per query head")
+    ap.add_argument("--shard", default=None, choices=["kv"],
+                    help="kv: ONE layer with its heads sharded over the --gpus ranks by KV group (strong scaling; one "
+                         "all-gather of the multiplier table per step) instead of one replica of the layer per rank")
     ap.add_argument("--sweep", default=None, choices=["length", "blocks", "chunks"],
                     help="speed sweeps on the Llama-3-8B shape instead of the benchmark line: input length at the "
                          "paper's B_h = 2048 tokens, or segment x block size at 128k")
@@ -750,6 +956,8 @@ def main():
         wl = synth.generator.with_(wl, fraction=args.fraction)
     if args.impl == "reference":
         run_reference(args, wl)
+    elif args.shard == "kv":
+        run_shard_kv(args, wl)
     else:
         run_ours(args, wl)
 

@@ -170,7 +170,13 @@ typedef enum ei_flags {
      and one O in tensor memory, Q.K^T three key blocks ahead of P.V, two sets of softmax warps on alternate key
      blocks that pass the row reference maxima to each other through shared memory; a CTA runs through several
      consecutive tiles of a segment.                                                                          */
-  EI_FLAG_ATTN_TRI = 1u << 12
+  EI_FLAG_ATTN_TRI = 1u << 12,
+  /* The plan holds a SHARD of the heads of a layer (whole KV groups; the other heads live in plans on other
+     GPUs): in TOTAL mode its index buffer is sized for all causal blocks of its heads, because the common total
+     is apportioned over the multipliers of ALL heads and a shard may be handed more than its own share.  Such a
+     plan is driven by ei_plan_observe, ei_stage_multipliers, (all-gather of the tables), ei_stage_apportion,
+     ei_stage_select instead of ei_plan.                                                                     */
+  EI_FLAG_HEAD_SHARD = 1u << 13
 } ei_flags;
 
 /* Fills *p with the paper's constants (e_t 1e-5, alpha 0.5, delta_t 0.4, cap 3, B_h 2048,
@@ -248,6 +254,30 @@ int ei_prefill_varlen(ei_plan_t* plan, const void* q, const void* k, const void*
 int ei_stage_pool(ei_plan_t* plan, const void* q, const void* k, void* stream);   /* Alg. 1     */
 int ei_stage_observe(ei_plan_t* plan, void* stream);   /* Alg. 2 + entropy, from the pooled reps */
 int ei_stage_budget(ei_plan_t* plan, void* stream);    /* Alg. 3 + block counts, from entropy    */
+/* Stages 1a + 1b of ei_plan alone (pooling and observation in the plan's schedule): ENTROPY and SCORES.  */
+int ei_plan_observe(ei_plan_t* plan, const void* q, const void* k, void* stream);
+/* Alg. 3 in its two halves, for a layer whose heads are sharded over several GPUs (one plan per shard, each
+   holding whole KV groups; everything of the method is per head except TOTAL mode's common total, which
+   couples the heads through the base budget b*):
+     ei_stage_multipliers   class and multiplier recurrence of the plan's heads from ENTROPY: CLASS and
+                            MULTIPLIERS (M = floor(m*4096 + 0.5), int32 [H, C_S]); when multipliers_out_dev is
+                            not NULL the table is also copied there (device, H*C_S int32) -- the send buffer of
+                            the all-gather;
+     ei_stage_apportion     block counts of the plan's heads as rows [first_head, first_head + H) of the
+                            apportionment of total_all blocks over the n_heads_all heads of
+                            multipliers_all_dev (device, int32 [n_heads_all, C_S], the gathered tables in head
+                            order): the same b*, the same leftover cells as one plan over all heads would find,
+                            so the shards' BUDGET rows are the rows of that plan bit for bit.  BASE mode looks
+                            at the plan's own rows only.  Writes BUDGET, OFFSETS and STATS (total and extremes
+                            of the plan's own heads; b* and leftover of the whole layer).
+   Between the two the caller gathers the tables (e.g. ncclAllGather on the same stream); no other exchange is
+   needed.  ei_stage_apportion fails with EI_ERR_BUDGET_INFEASIBLE when total_all is below the forced diagonal
+   blocks or above all causal blocks of n_heads_all heads, with EI_ERR_PLAN_MISMATCH when the plan's index
+   buffer could not hold what it may be handed (create it with EI_FLAG_HEAD_SHARD).  Asynchronous.
+   (Related Work: every quantity of the method is per head h; Alg. 3.)                                       */
+int ei_stage_multipliers(ei_plan_t* plan, int32_t* multipliers_out_dev, void* stream);
+int ei_stage_apportion(ei_plan_t* plan, const int32_t* multipliers_all_dev, int n_heads_all, int first_head,
+                       int64_t total_all, void* stream);
 int ei_stage_select(ei_plan_t* plan, void* stream);    /* top-k lists, from scores + counts      */
 
 typedef enum ei_item {
@@ -269,7 +299,8 @@ typedef enum ei_item {
      (H_kv of them instead of H); ENTROPY and SCORES stay per query head, and the aggregated tables that
      stages 2 and 3 read are:                                                                    */
   EI_ITEM_GROUP_ENTROPY = 11, /* float [H_kv, C_S]                                              */
-  EI_ITEM_GROUP_SCORES = 12   /* float [H_kv, sum_i C_i] ln A_g                                 */
+  EI_ITEM_GROUP_SCORES = 12,  /* float [H_kv, sum_i C_i] ln A_g                                 */
+  EI_ITEM_MULTIPLIERS = 13    /* int32 [H, C_S] (list heads): M = floor(m*4096 + 0.5) of Alg. 3     */
 } ei_item;
 
 /* Borrowed device pointer and size in bytes of one plan item; valid until ei_plan_destroy.    */

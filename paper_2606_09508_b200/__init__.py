@@ -26,6 +26,7 @@ from .binding import (  # noqa: F401
     FLAG_ATTN_QUAD,
     FLAG_ATTN_SPLIT,
     FLAG_ATTN_TRI,
+    FLAG_HEAD_SHARD,
     ROPE_NO_POOL,
     entropy_noalloc,
     lib,

@@ -41,7 +41,7 @@ class EiCompressParams(C.Structure):
 STATUS = dict(OK=0, INVALID_ARG=-1, UNSUPPORTED_SHAPE=-2, BUDGET_INFEASIBLE=-3, ARCH=-4, ALLOC=-5,
               CUDA=-6, DEVICE_TIMEOUT=-7, PLAN_MISMATCH=-8, NOT_PLANNED=-9, SCRATCH_TOO_SMALL=-10, WRONG_DEVICE=-11)
 ITEM = dict(GROUP_ENTROPY=11, GROUP_SCORES=12, ENTROPY=0, CLASS=1, BUDGET=2, OFFSETS=3, INDICES=4, SCORES=5, QMAX=6, QMIN=7, KMAX=8,
-            KMIN=9, STATS=10)
+            KMIN=9, STATS=10, MULTIPLIERS=13)
 BUDGET_BASE_TOKENS, BUDGET_TOTAL_FRACTION = 0, 1
 ROPE_NO_POOL = 1
 FLAG_ATTN_P_VIA_SMEM = 1
@@ -57,6 +57,7 @@ FLAG_ATTN_SKIP_ZERO_PV = 512
 FLAG_ATTN_QUAD = 1024
 FLAG_ATTN_SPLIT = 2048
 FLAG_ATTN_TRI = 4096
+FLAG_HEAD_SHARD = 8192
 
 # every symbol the header declares: (name, restype, argtypes)
 _P = C.c_void_p
@@ -73,6 +74,9 @@ SYMBOLS = [
     ("ei_stage_pool", C.c_int, [_P, _P, _P, _P]),
     ("ei_stage_observe", C.c_int, [_P, _P]),
     ("ei_stage_budget", C.c_int, [_P, _P]),
+    ("ei_plan_observe", C.c_int, [_P, _P, _P, _P]),
+    ("ei_stage_multipliers", C.c_int, [_P, _P, _P]),
+    ("ei_stage_apportion", C.c_int, [_P, _P, C.c_int, C.c_int, C.c_int64, _P]),
     ("ei_stage_select", C.c_int, [_P, _P]),
     ("ei_plan_get", C.c_int, [_P, C.c_int, C.POINTER(_P), C.POINTER(C.c_size_t)]),
     ("ei_plan_read", C.c_int, [_P, C.c_int, _P, C.c_size_t, _P]),
@@ -151,7 +155,7 @@ def params_default(H, Hkv, d, N, L_S, L_B, fraction=0.0) -> EiParams:
 
 _ITEM_DTYPE = {"GROUP_ENTROPY": np.float32, "GROUP_SCORES": np.float32, "ENTROPY": np.float32, "CLASS": np.uint8, "BUDGET": np.int32, "OFFSETS": np.int32,
                "INDICES": np.int32, "SCORES": np.float32, "QMAX": np.uint16, "QMIN": np.uint16,
-               "KMAX": np.uint16, "KMIN": np.uint16, "STATS": np.int64}
+               "KMAX": np.uint16, "KMIN": np.uint16, "STATS": np.int64, "MULTIPLIERS": np.int32}
 
 
 def _dev_ptr(t) -> int:
@@ -275,6 +279,20 @@ class Plan:
 
     def stage_budget(self, stream=None):
         _check(lib().ei_stage_budget(self._h, _stream_ptr(stream)), "ei_stage_budget")
+
+    # ---- a layer's heads sharded over several plans (one per GPU)
+    def observe(self, q, k, stream=None):
+        """Stages 1a + 1b alone."""
+        _check(lib().ei_plan_observe(self._h, _dev_ptr(q), _dev_ptr(k), _stream_ptr(stream)), "ei_plan_observe")
+
+    def stage_multipliers(self, out=None, stream=None):
+        """Alg. 3's classes and multipliers; `out`: an int32 device tensor [H, C_S] that also receives the table."""
+        _check(lib().ei_stage_multipliers(self._h, _dev_ptr(out), _stream_ptr(stream)), "ei_stage_multipliers")
+
+    def stage_apportion(self, multipliers_all, n_heads_all: int, first_head: int, total_all: int, stream=None):
+        """Block counts of this plan's heads from the gathered tables of all heads (device int32 [n_heads_all, C_S])."""
+        _check(lib().ei_stage_apportion(self._h, _dev_ptr(multipliers_all), int(n_heads_all), int(first_head),
+                                        int(total_all), _stream_ptr(stream)), "ei_stage_apportion")
 
     def stage_select(self, stream=None):
         _check(lib().ei_stage_select(self._h, _stream_ptr(stream)), "ei_stage_select")

@@ -127,6 +127,7 @@ Item item_of(const ei_plan_t* pl, int item) {
     case EI_ITEM_OFFSETS: return {pl->offsets, sizeof(int) * (size_t)(ls.cells + 1)};
     case EI_ITEM_GROUP_ENTROPY: return {pl->g_entropy, sizeof(float) * (size_t)ls.cells};
     case EI_ITEM_GROUP_SCORES: return {pl->g_scores, sizeof(float) * (size_t)ls.H * (size_t)ls.SC};
+    case EI_ITEM_MULTIPLIERS: return {pl->Mfx, sizeof(int) * (size_t)ls.cells};
     case EI_ITEM_INDICES: return {pl->indices, sizeof(int) * (size_t)pl->capacity};
     case EI_ITEM_SCORES: return {pl->scores, sizeof(float) * (size_t)s.H * (size_t)s.SC};
     case EI_ITEM_QMAX: return {pl->qmax, 2 * (size_t)s.cells * s.d};
@@ -159,7 +160,8 @@ int derive(ei_plan_t* pl, const ei_params* params, Shape s) {
     const int c_last = ei::causal_blocks(ls, ls.C_S - 1);
     const long long forced = (long long)ls.H * ((long long)ls.r * (ls.C_S - 1) + (c_last < ls.r ? c_last : ls.r));  // sum of min(r, C_i)
     if (T < forced || T > lall) return EI_ERR_BUDGET_INFEASIBLE;
-    need = T;
+    // a plan that holds a shard of a layer's heads can be handed more than its own share of a common total
+    need = (params->flags & EI_FLAG_HEAD_SHARD) ? lall : T;
   } else {
     if (!(params->base_budget_tokens > 0.0)) return EI_ERR_INVALID_ARG;
     const double base_blocks = params->base_budget_tokens / (double)s.L_B;
@@ -332,21 +334,60 @@ int ei_stage_observe(ei_plan_t* pl, void* stream) {
   return e == cudaSuccess ? EI_OK : EI_ERR_CUDA;
 }
 
-int ei_stage_budget(ei_plan_t* pl, void* stream) {
-  if (!pl) return EI_ERR_INVALID_ARG;
-  if (!on_plan_device(pl)) return EI_ERR_WRONG_DEVICE;
+namespace {
+int run_budget(ei_plan_t* pl, int phase, const int* m_all, int n_heads_all, int first_head, long long total_all,
+               void* stream) {
   ei::BudgetArgs a;
   a.mode = pl->params.budget_mode;
-  a.T = pl->T;
+  a.T = total_all;
   a.b_fx_base = pl->b_fx_base;
   a.e_t = pl->params.entropy_threshold;
   a.alpha = pl->params.alpha;
   a.delta_t = pl->params.delta_t;
   a.max_mult = pl->params.max_mult;
-  cudaError_t e = ei::launch_budget(pl->lshape, a, pl->group ? pl->g_entropy : pl->entropy, pl->rigid, pl->Mfx,
+  a.phase = phase;
+  a.H_all = n_heads_all;
+  a.first_head = first_head;
+  cudaError_t e = ei::launch_budget(pl->lshape, a, pl->group ? pl->g_entropy : pl->entropy, pl->rigid, pl->Mfx, m_all,
                                     pl->kblocks, pl->offsets, pl->stats, (cudaStream_t)stream);
   pl->launches += 1;
   return e == cudaSuccess ? EI_OK : EI_ERR_CUDA;
+}
+}  // namespace
+
+int ei_stage_budget(ei_plan_t* pl, void* stream) {
+  if (!pl) return EI_ERR_INVALID_ARG;
+  if (!on_plan_device(pl)) return EI_ERR_WRONG_DEVICE;
+  return run_budget(pl, ei::EI_BUDGET_PHASE_ALL, nullptr, pl->lshape.H, 0, pl->T, stream);
+}
+
+int ei_stage_multipliers(ei_plan_t* pl, int32_t* multipliers_out_dev, void* stream) {
+  if (!pl) return EI_ERR_INVALID_ARG;
+  if (!on_plan_device(pl)) return EI_ERR_WRONG_DEVICE;
+  int rc = run_budget(pl, ei::EI_BUDGET_PHASE_MULTIPLIERS, nullptr, pl->lshape.H, 0, pl->T, stream);
+  if (rc == EI_OK && multipliers_out_dev &&
+      cudaMemcpyAsync(multipliers_out_dev, pl->Mfx, sizeof(int) * (size_t)pl->lshape.cells, cudaMemcpyDeviceToDevice,
+                      (cudaStream_t)stream) != cudaSuccess)
+    rc = EI_ERR_CUDA;
+  return rc;
+}
+
+int ei_stage_apportion(ei_plan_t* pl, const int32_t* multipliers_all_dev, int n_heads_all, int first_head,
+                       int64_t total_all, void* stream) {
+  if (!pl || !multipliers_all_dev || n_heads_all <= 0 || first_head < 0) return EI_ERR_INVALID_ARG;
+  if (!on_plan_device(pl)) return EI_ERR_WRONG_DEVICE;
+  const ei::Shape& ls = pl->lshape;
+  if (first_head + ls.H > n_heads_all) return EI_ERR_INVALID_ARG;
+  if ((long long)n_heads_all * ls.C_S > (1 << 20)) return EI_ERR_UNSUPPORTED_SHAPE;  // one CTA walks every cell
+  if (pl->params.budget_mode == EI_BUDGET_TOTAL_FRACTION) {
+    const int c_last = ei::causal_blocks(ls, ls.C_S - 1);
+    const long long forced1 = (long long)ls.r * (ls.C_S - 1) + (c_last < ls.r ? c_last : ls.r);  // sum of min(r, C_i)
+    if (total_all < forced1 * n_heads_all || total_all > (long long)ls.SC * n_heads_all) return EI_ERR_BUDGET_INFEASIBLE;
+    // budget flows between the shards: mine may get anything up to all causal blocks of its heads
+    const long long all_mine = (long long)ls.H * ls.SC;
+    if (pl->capacity < (total_all < all_mine ? total_all : all_mine)) return EI_ERR_PLAN_MISMATCH;
+  }
+  return run_budget(pl, ei::EI_BUDGET_PHASE_APPORTION, multipliers_all_dev, n_heads_all, first_head, total_all, stream);
 }
 
 int ei_stage_select(ei_plan_t* pl, void* stream) {
@@ -363,8 +404,7 @@ int ei_stage_select(ei_plan_t* pl, void* stream) {
   return e == cudaSuccess ? EI_OK : EI_ERR_CUDA;
 }
 
-int ei_plan(ei_plan_t* pl, const void* q, const void* k, const void* v, void* stream) {
-  (void)v;
+int ei_plan_observe(ei_plan_t* pl, const void* q, const void* k, void* stream) {
   if (!pl || !q || !k) return EI_ERR_INVALID_ARG;
   if (!on_plan_device(pl)) return EI_ERR_WRONG_DEVICE;
   int rc;
@@ -391,6 +431,12 @@ int ei_plan(ei_plan_t* pl, const void* q, const void* k, const void* v, void* st
     rc = ei_stage_pool(pl, q, k, stream);
     if (rc == EI_OK) rc = ei_stage_observe(pl, stream);
   }
+  return rc;
+}
+
+int ei_plan(ei_plan_t* pl, const void* q, const void* k, const void* v, void* stream) {
+  (void)v;
+  int rc = ei_plan_observe(pl, q, k, stream);
   if (rc == EI_OK) rc = ei_stage_budget(pl, stream);
   if (rc == EI_OK) rc = ei_stage_select(pl, stream);
   return rc;

@@ -75,9 +75,14 @@ struct BudgetArgs {
   long long T;         // TOTAL mode target
   long long b_fx_base; // BASE mode base budget, 1/4096 block
   double e_t, alpha, delta_t, max_mult;
+  int phase;           // EI_BUDGET_PHASE_*
+  int H_all;           // heads the apportionment runs over (the plan's own unless the layer is sharded)
+  int first_head;      // where this plan's heads sit among them
 };
+enum { EI_BUDGET_PHASE_ALL = 0, EI_BUDGET_PHASE_MULTIPLIERS = 1, EI_BUDGET_PHASE_APPORTION = 2 };
+// Mall: the multiplier table [H_all, C_S] of EI_BUDGET_PHASE_APPORTION (device; otherwise unused)
 cudaError_t launch_budget(const Shape& s, const BudgetArgs& a, const float* entropy,
-                          unsigned char* rigid, int* Mfx, int* kblocks, int* offsets, Stats* stats,
+                          unsigned char* rigid, int* Mfx, const int* Mall, int* kblocks, int* offsets, Stats* stats,
                           cudaStream_t st);
 
 // items (may be null): the stage-4 records of every (cell, tile pair), written by the warp that made the cell's list

@@ -763,6 +763,11 @@ cudaError_t launch_group_aggregate(const Shape& s, const float* scores, const fl
 // BASE mode: b = base budget.  TOTAL mode: b* = largest b with sum_c k(c,b) <= T, found by
 // bisection (each thread keeps its few cells in registers); the R = T - sum k(c,b*) leftover blocks go to the first
 // R cells, in increasing c, whose count grows at b*+1.  Offsets are the exclusive scan of k.
+//
+// The kernel runs in one piece or in its two halves (a.phase): the multipliers alone (A), and the apportionment
+// alone (B, C) over a table of multipliers that may cover MORE heads than this plan holds -- the heads of a layer
+// sharded over several GPUs, whose tables were gathered: every shard then finds the same b* and the same
+// leftover cells for all H_all heads and keeps the counts of its own heads [first_head, first_head + H).
 // =================================================================================================
 constexpr int BUD_THREADS = 1024;
 
@@ -805,23 +810,29 @@ __device__ long long block_excl_scan(long long v, long long* warp_sums, long lon
 
 __global__ void __launch_bounds__(BUD_THREADS, 1)
 budget_kernel(Shape s, BudgetArgs a, const float* __restrict__ entropy, unsigned char* __restrict__ rigid,
-              int* __restrict__ Mfx, int* __restrict__ kblocks, int* __restrict__ offsets,
+              int* __restrict__ Mfx, const int* Mall, int* __restrict__ kblocks, int* __restrict__ offsets,
               Stats* __restrict__ stats) {
   __shared__ long long s_warp[33];
   __shared__ int s_rigid, s_mink, s_maxk;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int cells = (int)s.cells;
+  // the apportionment runs over the cells of all a.H_all heads; mine are [cell_lo, cell_hi)
+  const int cells = a.H_all * s.C_S;
+  const int cell_lo = a.first_head * s.C_S, cell_hi = cell_lo + (int)s.cells;
   if (tid == 0) {
     s_rigid = 0;
     s_mink = 0x7fffffff;
     s_maxk = 0;
   }
   __syncthreads();
+  if (a.phase == EI_BUDGET_PHASE_APPORTION) {  // the classes were made by an earlier launch: count them for the statistics
+    for (int h = tid; h < s.H; h += BUD_THREADS)
+      if (rigid[h]) atomicAdd(&s_rigid, 1);
+  }
 
   // ---- A: class + multiplier recurrence, one warp per head -------------------------------------------
   // The division-heavy increments are computed lane-parallel; only add / clamp is sequential.  Every
   // lane carries the same running multiplier, so lane t keeps the value after step t of its chunk.
-  for (int h = warp; h < s.H; h += BUD_THREADS / 32) {
+  for (int h = warp; h < s.H && a.phase != EI_BUDGET_PHASE_APPORTION; h += BUD_THREADS / 32) {
     const float* e = entropy + (long long)h * s.C_S;
     double emax = -INFINITY;
     for (int i = lane; i < s.C_S; i += 32) emax = fmax(emax, (double)e[i]);
@@ -863,6 +874,8 @@ budget_kernel(Shape s, BudgetArgs a, const float* __restrict__ entropy, unsigned
     }
   }
   __syncthreads();
+  if (a.phase == EI_BUDGET_PHASE_MULTIPLIERS) return;  // (block-uniform)
+  const int* Mt = a.phase == EI_BUDGET_PHASE_APPORTION ? Mall : Mfx;  // the table the apportionment runs over
 
   // ---- B: base budget: plain bisection, every thread evaluating its own few cells per round ------
   const int cpt = (cells + BUD_THREADS - 1) / BUD_THREADS;
@@ -873,7 +886,7 @@ budget_kernel(Shape s, BudgetArgs a, const float* __restrict__ entropy, unsigned
 #pragma unroll
   for (int t = 0; t < CACHE; ++t) {
     const int c = c0 + t;
-    Mreg[t] = (c < c1) ? Mfx[c] : 0;
+    Mreg[t] = (c < c1) ? Mt[c] : 0;
     Creg[t] = (c < c1) ? causal_blocks(s, (i_first + t) % s.C_S) : 0;
   }
   __shared__ int s_part[32];
@@ -895,7 +908,7 @@ budget_kernel(Shape s, BudgetArgs a, const float* __restrict__ entropy, unsigned
       for (int u = 0; u < CACHE; ++u)
         if (c0 + u < c1) t += kc(Mreg[u], Creg[u]);
     } else {
-      for (int c = c0, i = i_first; c < c1; ++c, i = (i + 1 == s.C_S ? 0 : i + 1)) t += kc(Mfx[c], causal_blocks(s, i));
+      for (int c = c0, i = i_first; c < c1; ++c, i = (i + 1 == s.C_S ? 0 : i + 1)) t += kc(Mt[c], causal_blocks(s, i));
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
@@ -930,9 +943,9 @@ budget_kernel(Shape s, BudgetArgs a, const float* __restrict__ entropy, unsigned
   long long base_sum = 0, grow_cnt = 0;
   for (int c = c0, i = i_first; c < c1; ++c, i = (i + 1 == s.C_S ? 0 : i + 1)) {
     const int Ci = causal_blocks(s, i);
-    const long long k0 = cell_blocks(Mfx[c], bstar, s.r, Ci);
+    const long long k0 = cell_blocks(Mt[c], bstar, s.r, Ci);
     base_sum += k0;
-    if (a.mode == EI_BUDGET_TOTAL_FRACTION) grow_cnt += cell_blocks(Mfx[c], bstar + 1, s.r, Ci) > k0;
+    if (a.mode == EI_BUDGET_TOTAL_FRACTION) grow_cnt += cell_blocks(Mt[c], bstar + 1, s.r, Ci) > k0;
   }
   long long total0, dummy;
   block_excl_scan(base_sum, s_warp, &total0);
@@ -943,29 +956,31 @@ budget_kernel(Shape s, BudgetArgs a, const float* __restrict__ entropy, unsigned
   int kmin = 0x7fffffff, kmax = 0;
   for (int c = c0, i = i_first; c < c1; ++c, i = (i + 1 == s.C_S ? 0 : i + 1)) {
     const int Ci = causal_blocks(s, i);
-    long long kc = cell_blocks(Mfx[c], bstar, s.r, Ci);
-    if (a.mode == EI_BUDGET_TOTAL_FRACTION && cell_blocks(Mfx[c], bstar + 1, s.r, Ci) > kc) {
+    long long kc = cell_blocks(Mt[c], bstar, s.r, Ci);
+    if (a.mode == EI_BUDGET_TOTAL_FRACTION && cell_blocks(Mt[c], bstar + 1, s.r, Ci) > kc) {
       if (grow_before < R) kc += 1;
       grow_before += 1;
     }
-    kblocks[c] = (int)kc;
-    my_sum += kc;
-    kmin = min(kmin, (int)kc);
-    kmax = max(kmax, (int)kc);
+    if (c >= cell_lo && c < cell_hi) {
+      kblocks[c - cell_lo] = (int)kc;
+      my_sum += kc;
+      kmin = min(kmin, (int)kc);
+      kmax = max(kmax, (int)kc);
+    }
   }
   long long total1;
   long long off = block_excl_scan(my_sum, s_warp, &total1);
-  for (int c = c0; c < c1; ++c) {
-    offsets[c] = (int)off;
-    off += kblocks[c];
+  for (int c = max(c0, cell_lo); c < min(c1, cell_hi); ++c) {
+    offsets[c - cell_lo] = (int)off;
+    off += kblocks[c - cell_lo];
   }
-  if (c0 < c1) {
+  if (kmax > 0) {
     atomicMin(&s_mink, kmin);
     atomicMax(&s_maxk, kmax);
   }
   __syncthreads();
   if (tid == 0) {
-    offsets[cells] = (int)total1;
+    offsets[cell_hi - cell_lo] = (int)total1;
     stats->total = total1;
     stats->rigid_heads = s_rigid;
     stats->b_star = bstar;
@@ -978,8 +993,8 @@ budget_kernel(Shape s, BudgetArgs a, const float* __restrict__ entropy, unsigned
 }
 
 cudaError_t launch_budget(const Shape& s, const BudgetArgs& a, const float* entropy, unsigned char* rigid,
-                          int* Mfx, int* kblocks, int* offsets, Stats* stats, cudaStream_t st) {
-  budget_kernel<<<1, BUD_THREADS, 0, st>>>(s, a, entropy, rigid, Mfx, kblocks, offsets, stats);
+                          int* Mfx, const int* Mall, int* kblocks, int* offsets, Stats* stats, cudaStream_t st) {
+  budget_kernel<<<1, BUD_THREADS, 0, st>>>(s, a, entropy, rigid, Mfx, Mall, kblocks, offsets, stats);
   return cudaGetLastError();
 }
 
