@@ -851,6 +851,59 @@ def run_chunk_sweep(args, ei, torch, wl):
                           "steps": args.steps}), flush=True)
 
 
+def run_varlen(args):
+    """A packed batch of many short sequences (64 x 2048 tokens, Llama-3-8B heads, L_S 256 / L_B 128, half of each
+    sequence's causal blocks): ei_prefill_varlen in one set of five launches against one ei_plan +
+    ei_sparse_prefill per sequence (what a batch cost before; still what group-shared lists and the other kernels do)."""
+    import torch
+
+    import paper_2606_09508_b200 as ei
+    Hq, Hkv, d, L_S, L_B, n_seq, n_tok, f = 32, 8, 128, 256, 128, 64, 2048, 0.5
+    total = n_seq * n_tok
+    q, k, v = synth.generate_plain(Hq, Hkv, total, d, seed=4242)
+
+    def dev(b):
+        return torch.from_numpy(b.view(np.int16)).cuda().view(torch.bfloat16)
+    qd, kd, vd = dev(q), dev(k), dev(v)
+    out_a, out_b = torch.zeros_like(qd), torch.zeros_like(qd)
+    cu = np.arange(n_seq + 1, dtype=np.int32) * n_tok
+    pa = ei.params_default(Hq, Hkv, d, total, L_S, L_B, f)         # room for all sequences' tables side by side
+    plan_a = ei.Plan(pa)
+    pb = ei.params_default(Hq, Hkv, d, n_tok, L_S, L_B, f)           # one sequence at a time
+    pb.q_stride_head = pb.k_stride_head = pb.v_stride_head = pb.o_stride_head = total * d
+    plan_b = ei.Plan(pb)
+    stream = torch.cuda.current_stream()
+
+    def packed():
+        plan_a.prefill_varlen(qd, kd, vd, out_a, cu)
+
+    def loop():
+        for b in range(n_seq):
+            lo, hi = b * n_tok, (b + 1) * n_tok
+            plan_b.plan(qd[:, lo:hi], kd[:, lo:hi])
+            plan_b.sparse_prefill(qd[:, lo:hi], kd[:, lo:hi], vd[:, lo:hi], out_b[:, lo:hi])
+    res = {}
+    for name, fn, pl in (("one_set_of_launches", packed, plan_a), ("per_sequence_loop", loop, plan_b)):
+        for _ in range(max(args.warmup, 3)):
+            fn()
+        torch.cuda.synchronize()
+        l0 = pl.launches()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.steps):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if pl.status() != 0:
+            raise RuntimeError("device-side wait timed out")
+        res[name] = {"ms_per_batch": e0.elapsed_time(e1) / args.steps, "launches_per_batch": (pl.launches() - l0) // args.steps}
+    same = bool(torch.equal(out_a.view(torch.int16), out_b.view(torch.int16)))
+    print(json.dumps({"sweep": "varlen", "batch": f"{n_seq} x {n_tok} tokens", "heads": [Hq, Hkv], "head_dim": d,
+                      "segment_len": L_S, "block_len": L_B, "budget_fraction": f, **res,
+                      "speedup": res["per_sequence_loop"]["ms_per_batch"] / res["one_set_of_launches"]["ms_per_batch"],
+                      "outputs_identical": same}))
+
+
 def run_sweep(args):
     import torch
 
@@ -944,10 +997,13 @@ def main():
     ap.add_argument("--shard", default=None, choices=["kv"],
                     help="kv: ONE layer with its heads sharded over the --gpus ranks by KV group (strong scaling; one "
                          "all-gather of the multiplier table per step) instead of one replica of the layer per rank")
-    ap.add_argument("--sweep", default=None, choices=["length", "blocks", "chunks"],
+    ap.add_argument("--sweep", default=None, choices=["length", "blocks", "chunks", "varlen"],
                     help="speed sweeps on the Llama-3-8B shape instead of the benchmark line: input length at the "
                          "paper's B_h = 2048 tokens, or segment x block size at 128k")
     args = ap.parse_args()
+    if args.sweep == "varlen":
+        run_varlen(args)
+        return
     if args.sweep:
         run_sweep(args)
         return

@@ -245,7 +245,17 @@ int ei_plan_pooled(ei_plan_t* plan, void* stream);
    when a sequence does not fit (EI_ERR_PLAN_MISMATCH), when in TOTAL mode the fraction of a short sequence's
    blocks is below its forced diagonal blocks (EI_ERR_BUDGET_INFEASIBLE; BASE mode has no such limit) or when
    cu_seqlens is not monotone (EI_ERR_INVALID_ARG).
-   Asynchronous; afterwards the plan is targeted at, and holds the tables of, the last non-empty sequence.   */
+   Launches: sequences whose tables fit the plan's side by side (cells, scores, K representatives, list
+   entries: a plan created for the batch's total length, each sequence rounded up to whole segments, holds them
+   all; at most 256 at a time) run in ONE set of five launches -- pooling, observation, budget (one CTA per
+   sequence), selection, attention -- in which every CTA looks up its sequence in a small table copied to the
+   device with the call; this applies to head_dim 128, block_len 128, segments a multiple of 256, per-head lists
+   and the default attention kernel.  A sequence that fits only on its own (a plan made for the longest sequence),
+   and every sequence under group-shared lists, the other kernels or other shapes, takes the plan re-targeted to
+   it and the ordinary two calls (four to five launches per sequence).  The results are the same either way.
+   Asynchronous; afterwards the plan is targeted at the last non-empty sequence.  It holds that sequence's
+   tables when the sequence ran on its own; after a set of packed launches the tables hold the batch, one
+   sequence after another, and ei_sparse_prefill returns EI_ERR_NOT_PLANNED until the next ei_plan.          */
 int ei_prefill_varlen(ei_plan_t* plan, const void* q, const void* k, const void* v, void* out,
                       const int32_t* cu_seqlens_host, int n_seqs, void* stream);
 

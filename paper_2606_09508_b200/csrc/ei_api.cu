@@ -36,6 +36,7 @@ struct ei_plan_s {
   ei::Stats* stats;
   int* status;
   int* sched;  // item counter of the persistent attention kernel
+  ei::PackedSeq* pk;  // per-sequence table of a packed batch that runs in one set of launches (MAX_PACKED entries)
   int* items;  // per (list cell, tile pair) records for stage 4, rebuilt when the lists change
   bool items_valid;
   int device;  // the device the plan's storage lives on
@@ -242,7 +243,7 @@ void ei_plan_destroy(ei_plan_t* pl) {
   if (!pl) return;
   void* ptrs[] = {pl->entropy, pl->rigid, pl->Mfx, pl->kblocks, pl->offsets, pl->indices, pl->scores, pl->qmax,
                   pl->qmin, pl->kmax, pl->kmin, pl->stats, pl->status, pl->sq, pl->sk, pl->sv, pl->so,
-                  pl->g_entropy, pl->g_scores, pl->sched, pl->items};
+                  pl->g_entropy, pl->g_scores, pl->sched, pl->items, pl->pk};
   for (void* p : ptrs)
     if (p) cudaFree(p);
   for (int g = 0; pl->sub && g < pl->shape.Hkv; ++g)
@@ -291,13 +292,14 @@ int ei_plan_create(const ei_params* params, ei_plan_t** out) {
   pl->cap_lscores = lall;
   pl->capacity = pl->need_idx;
 
-  bool ok = dalloc(&pl->entropy, (size_t)s.cells) && dalloc(&pl->rigid, (size_t)ls.H) &&
+  bool ok = dalloc(&pl->entropy, (size_t)s.cells) && dalloc(&pl->rigid, (size_t)ls.H * ei::MAX_PACKED) &&
+            dalloc(&pl->pk, (size_t)ei::MAX_PACKED) &&
             dalloc(&pl->Mfx, (size_t)ls.cells) && dalloc(&pl->kblocks, (size_t)ls.cells) &&
-            dalloc(&pl->offsets, (size_t)ls.cells + 1) && dalloc(&pl->indices, (size_t)pl->capacity) &&
+            dalloc(&pl->offsets, (size_t)ls.cells + ei::MAX_PACKED) && dalloc(&pl->indices, (size_t)pl->capacity) &&
             (!pl->group || (dalloc(&pl->g_entropy, (size_t)ls.cells) && dalloc(&pl->g_scores, (size_t)lall))) &&
             dalloc(&pl->scores, (size_t)all) && dalloc(&pl->qmax, (size_t)s.cells * s.d) &&
             dalloc(&pl->qmin, (size_t)s.cells * s.d) && dalloc(&pl->kmax, (size_t)s.Hkv * s.C_B * s.d) &&
-            dalloc(&pl->kmin, (size_t)s.Hkv * s.C_B * s.d) && dalloc(&pl->stats, 1) && dalloc(&pl->status, 4) &&
+            dalloc(&pl->kmin, (size_t)s.Hkv * s.C_B * s.d) && dalloc(&pl->stats, (size_t)ei::MAX_PACKED) && dalloc(&pl->status, 4) &&
             dalloc(&pl->sched, 2) && dalloc(&pl->items, (size_t)ls.cells * (s.L_S >= 256 ? s.L_S / 256 : 1) * 8);
   if (!ok) {
     ei_plan_destroy(pl);
@@ -739,6 +741,65 @@ int ei_plan_set_lengths(ei_plan_t* pl, int seq_len, int q_len, int k_blocks_vali
   return EI_OK;
 }
 
+namespace {
+// Can a packed batch run in one set of launches on this plan?  (The staged planning kernels and the default
+// stage-4 kernel take the per-sequence table; group-shared lists, the other attention kernels and the other
+// shapes go sequence by sequence.)
+bool packed_capable(const ei_plan_t* pl) {
+  const ei::Shape& s = pl->shape;
+  const uint32_t other = EI_FLAG_GROUP_SHARED | EI_FLAG_ATTN_SPLIT | EI_FLAG_ATTN_SKIP_ZERO_PV | EI_FLAG_ATTN_P_VIA_SMEM |
+                         EI_FLAG_ATTN_PAIR_8WARP | EI_FLAG_ATTN_PERSISTENT | EI_FLAG_ATTN_SINGLE_TILE | EI_FLAG_ATTN_TRI |
+                         EI_FLAG_ATTN_QUAD;
+  return s.L_S % 256 == 0 && s.d == 128 && s.L_B == 128 && !(pl->params.flags & other);
+}
+
+// sequences [b0, b1) of the batch (all non-empty, all fitting the plan's tables together) in five launches
+int run_packed(ei_plan_t* pl, const std::vector<ei::PackedSeq>& seqs_in, long long n_tokens, const void* q, const void* k,
+               const void* v, void* out, cudaStream_t st) {
+  std::vector<ei::PackedSeq> hp(seqs_in);
+  const int n = (int)hp.size();
+  ei::packed_fill_work(hp.data(), n);
+  if (cudaMemcpyAsync(pl->pk, hp.data(), sizeof(ei::PackedSeq) * n, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return EI_ERR_CUDA;
+  cudaError_t e = ei::launch_pool_packed(pl->pk, hp.data(), n, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, pl->qmax,
+                                         pl->qmin, pl->kmax, pl->kmin, st);
+  if (e == cudaSuccess)
+    e = ei::launch_observe_packed(pl->pk, hp.data(), n, pl->qmax, pl->qmin, pl->kmax, pl->kmin, pl->obs_scale, pl->scores,
+                                  pl->entropy, st);
+  ei::BudgetArgs a;
+  a.mode = pl->params.budget_mode;
+  a.T = 0;
+  a.b_fx_base = pl->b_fx_base;
+  a.e_t = pl->params.entropy_threshold;
+  a.alpha = pl->params.alpha;
+  a.delta_t = pl->params.delta_t;
+  a.max_mult = pl->params.max_mult;
+  a.phase = ei::EI_BUDGET_PHASE_ALL;
+  a.H_all = 0;
+  a.first_head = 0;
+  if (e == cudaSuccess)
+    e = ei::launch_budget_packed(pl->pk, n, a, pl->entropy, pl->rigid, pl->Mfx, pl->kblocks, pl->offsets, pl->stats, st);
+  if (e == cudaSuccess)
+    e = ei::launch_select_packed(pl->pk, hp.data(), n, pl->scores, pl->kblocks, pl->offsets, pl->indices, pl->items, st);
+  pl->launches += 4;
+  if (e != cudaSuccess) return EI_ERR_CUDA;
+  ei::AttnArgs at{};
+  at.q = (const __nv_bfloat16*)q;
+  at.k = (const __nv_bfloat16*)k;
+  at.v = (const __nv_bfloat16*)v;
+  at.out = (__nv_bfloat16*)out;
+  at.offsets = pl->offsets;
+  at.indices = pl->indices;
+  at.items = pl->items;
+  at.status = pl->status;
+  at.scale = (float)pl->attn_scale;
+  at.skip_log2 = (pl->params.flags & EI_FLAG_ATTN_NO_SKIP) ? INFINITY : 24.0f;
+  const int rc = ei::launch_attention_quad_packed(pl->pk, hp.data(), n, n_tokens, at, st);
+  pl->launches += 1;
+  return rc;
+}
+}  // namespace
+
 int ei_prefill_varlen(ei_plan_t* pl, const void* q, const void* k, const void* v, void* out,
                       const int32_t* cu_seqlens_host, int n_seqs, void* stream) {
   if (!pl || !q || !k || !v || !out || !cu_seqlens_host || n_seqs < 0) return EI_ERR_INVALID_ARG;
@@ -747,8 +808,12 @@ int ei_prefill_varlen(ei_plan_t* pl, const void* q, const void* k, const void* v
   if (cu[0] < 0) return EI_ERR_INVALID_ARG;
   for (int b = 0; b < n_seqs; ++b)
     if (cu[b + 1] < cu[b]) return EI_ERR_INVALID_ARG;
-  // every sequence has to fit the plan before anything is launched (host-only probes)
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return EI_ERR_UNSUPPORTED_SHAPE;
+  // every sequence has to fit the plan before anything is launched (host-only probes); what a plan of each
+  // sequence alone would look like is kept for the packed launches
   const ei_plan_t saved = *pl;
+  std::vector<ei::PackedSeq> seqs;
+  std::vector<long long> need;
   for (int b = 0; b < n_seqs; ++b) {
     const int len = cu[b + 1] - cu[b];
     if (len == 0) continue;
@@ -757,20 +822,72 @@ int ei_prefill_varlen(ei_plan_t* pl, const void* q, const void* k, const void* v
       *pl = saved;
       return rc;
     }
+    ei::PackedSeq P{};
+    P.s = pl->shape;
+    P.s.KB_cap = P.s.C_B;  // its K representatives are laid out as a plan of this sequence alone would lay them out
+    P.tok0 = cu[b];
+    P.T = pl->T;
+    P.index = b;  // (the batch position for now; the slot within its set of launches is assigned below)
+    seqs.push_back(P);
+    need.push_back(pl->need_idx);
   }
   const ei_params& p = pl->params;
-  for (int b = 0; b < n_seqs; ++b) {
-    const int len = cu[b + 1] - cu[b];
-    if (len == 0) continue;
-    int rc = ei_plan_set_lengths(pl, len, 0, 0);
-    const long long t0 = cu[b];
-    const __nv_bfloat16* qb = (const __nv_bfloat16*)q + t0 * p.q_stride_tok;
-    const __nv_bfloat16* kb = (const __nv_bfloat16*)k + t0 * p.k_stride_tok;
-    const __nv_bfloat16* vb = (const __nv_bfloat16*)v + t0 * p.v_stride_tok;
-    __nv_bfloat16* ob = (__nv_bfloat16*)out + t0 * p.o_stride_tok;
-    if (rc == EI_OK) rc = ei_plan(pl, qb, kb, vb, stream);
-    if (rc == EI_OK) rc = ei_sparse_prefill(pl, qb, kb, vb, ob, stream);
+  const bool packed_ok = packed_capable(pl) && ei::observe_shape_supported(pl->shape);
+  const long long n_tokens = cu[n_seqs];
+  const long long kreps_cap = (long long)saved.shape.Hkv * saved.shape.KB_cap;
+  cudaStream_t st = (cudaStream_t)stream;
+  size_t i0 = 0;
+  bool last_packed = false;
+  while (i0 < seqs.size()) {
+    // the longest run of sequences from i0 on whose tables fit the plan's side by side
+    size_t i1 = i0;
+    long long cells = 0, sc = 0, kb = 0, idx = 0;
+    std::vector<ei::PackedSeq> grp;
+    while (packed_ok && i1 < seqs.size() && (int)grp.size() < ei::MAX_PACKED) {
+      const ei::Shape& sb = seqs[i1].s;
+      if (cells + sb.cells > pl->cap_cells || sc + (long long)sb.H * sb.SC > pl->cap_scores ||
+          kb + (long long)sb.Hkv * sb.C_B > kreps_cap || idx + need[i1] > pl->capacity)
+        break;
+      ei::PackedSeq P = seqs[i1];
+      P.cell0 = cells;
+      P.off0 = cells + (long long)grp.size();
+      P.sc0 = sc;
+      P.kb0 = kb;
+      P.idx0 = idx;
+      P.head0 = (int)grp.size() * sb.H;
+      P.index = (int)grp.size();
+      grp.push_back(P);
+      cells += sb.cells;
+      sc += (long long)sb.H * sb.SC;
+      kb += (long long)sb.Hkv * sb.C_B;
+      idx += need[i1];
+      ++i1;
+    }
+    int rc;
+    if (grp.size() >= 2) {
+      rc = run_packed(pl, grp, n_tokens, q, k, v, out, st);
+      last_packed = true;
+    } else {  // one sequence on its own: the plan re-targeted to it, the ordinary two calls
+      i1 = i0 + 1;
+      const long long t0 = seqs[i0].tok0;
+      rc = ei_plan_set_lengths(pl, seqs[i0].s.N, 0, 0);
+      const __nv_bfloat16* qb = (const __nv_bfloat16*)q + t0 * p.q_stride_tok;
+      const __nv_bfloat16* kb1 = (const __nv_bfloat16*)k + t0 * p.k_stride_tok;
+      const __nv_bfloat16* vb = (const __nv_bfloat16*)v + t0 * p.v_stride_tok;
+      __nv_bfloat16* ob = (__nv_bfloat16*)out + t0 * p.o_stride_tok;
+      if (rc == EI_OK) rc = ei_plan(pl, qb, kb1, vb, stream);
+      if (rc == EI_OK) rc = ei_sparse_prefill(pl, qb, kb1, vb, ob, stream);
+      last_packed = false;
+    }
     if (rc != EI_OK) return rc;
+    i0 = i1;
+  }
+  if (!seqs.empty()) {
+    ei_plan_set_lengths(pl, seqs.back().s.N, 0, 0);  // left targeted at the last non-empty sequence
+    if (last_packed) {  // the tables hold a batch, not that sequence: nothing to attend from until the next ei_plan
+      pl->planned = false;
+      pl->items_valid = false;
+    }
   }
   return EI_OK;
 }

@@ -286,7 +286,8 @@ __global__ void __maxnreg__(96)
 sparse_attention_quad_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
                              const __grid_constant__ CUtensorMap tmv, __nv_bfloat16* __restrict__ out,
                              const int* __restrict__ items, const int* __restrict__ indices,
-                             int* __restrict__ status, Shape s, float scale_log2, float skip_log2) {
+                             int* __restrict__ status, Shape s, float scale_log2, float skip_log2,
+                             const PackedSeq* pk, int npk) {
   using L = QuadSmem<D, BN, NSLOT>;
   static_assert(BN == 128 && D == 128, "the quad-layout kernels are written for head_dim 128 and 128-wide key blocks");
   extern __shared__ unsigned char att_smem_raw[];
@@ -307,6 +308,16 @@ sparse_attention_quad_kernel(const __grid_constant__ CUtensorMap tmq, const __gr
 
   const int pairs_per_seg = s.L_S / (2 * QBM);
   int bid = blockIdx.x;
+  int tok0 = 0;  // a packed batch: my sequence starts here in q, k, v, out (the tensor maps span the whole batch)
+  if (pk != nullptr) {
+    const PackedSeq& P = pk[packed_find(pk, npk, bid, &PackedSeq::w_att)];
+    s = P.s;
+    bid -= P.w_att;
+    tok0 = (int)P.tok0;
+    items += P.cell0 * pairs_per_seg * 8;
+    indices += P.idx0;
+    out += P.tok0 * s.os_t;
+  }
   const int pr = bid % pairs_per_seg;
   bid /= pairs_per_seg;
   const int h = bid % s.H;
@@ -341,7 +352,7 @@ sparse_attention_quad_kernel(const __grid_constant__ CUtensorMap tmq, const __gr
       mbar_expect_tx(BAR(B_QFULL + t), L::Q_BYTES);
 #pragma unroll
       for (int p = 0; p < D / 64; ++p)
-        tma_load_3d(sQ + t * L::Q_BYTES + p * (QBM * 128), &tmq, p * 64, q0 + t * QBM, h, BAR(B_QFULL + t));
+        tma_load_3d(sQ + t * L::Q_BYTES + p * (QBM * 128), &tmq, p * 64, tok0 + q0 + t * QBM, h, BAR(B_QFULL + t));
     }
   }
   // my item's record: list offset, blocks visible to tile 0 / tile 1, first masked entry of either, first block
@@ -356,7 +367,7 @@ sparse_attention_quad_kernel(const __grid_constant__ CUtensorMap tmq, const __gr
     const CUtensorMap* tm = (u & 1) ? &tmv : &tmk;
 #pragma unroll
     for (int p = 0; p < D / 64; ++p)
-      tma_load_3d(sRing + slot * L::KV_BYTES + p * (BN * 128), tm, p * 64, blk * BN, g, BAR(B_FULL + slot));
+      tma_load_3d(sRing + slot * L::KV_BYTES + p * (BN * 128), tm, p * 64, tok0 + blk * BN, g, BAR(B_FULL + slot));
   };
   int issued = 0;
   // testing aid (ei_plan_debug_waits): one ring item the producer leaves out, so that a bounded wait runs out
@@ -1146,6 +1157,32 @@ cudaError_t launch_attention_items(const Shape& ls, const int* offsets, const in
   return cudaGetLastError();
 }
 
+// One launch over the sequences of a packed batch: the tensor maps span the whole packed tensors (n_tokens rows),
+// a CTA adds its sequence's first token to the row coordinates.  What lies behind a sequence's last row is the next
+// sequence's data instead of the zero fill a tensor's end gives: queries there are computed and not stored, keys
+// there lie above every row of the sequence and fall to the causal mask, their V rows meet P = 0.
+int launch_attention_quad_packed(const PackedSeq* pk, const PackedSeq* pk_host, int npk, long long n_tokens,
+                                 const AttnArgs& a, cudaStream_t st) {
+  constexpr int D = 128, BN = 128, NSLOT = 5;
+  using L = QuadSmem<D, BN, NSLOT>;
+  const Shape& s = pk_host[npk - 1].s;
+  if (!a.items || n_tokens <= 0) return EI_ERR_INVALID_ARG;
+  CUtensorMap tmq, tmk, tmv;
+  if (!make_tensor_map(&tmq, a.q, D, (int)n_tokens, s.H, s.qs_t, s.qs_h, QBM) ||
+      !make_tensor_map(&tmk, a.k, D, (int)n_tokens, s.Hkv, s.ks_t, s.ks_h, BN) ||
+      !make_tensor_map(&tmv, a.v, D, (int)n_tokens, s.Hkv, s.vs_t, s.vs_h, BN))
+    return EI_ERR_CUDA;
+  const long long grid = pk_host[npk - 1].w_att + (long long)s.H * s.C_S * (s.L_S / (2 * QBM));
+  const float scale_log2 = a.scale * 1.4426950408889634f;
+  const bool skip = a.skip_log2 < INFINITY;
+  auto kern = skip ? sparse_attention_quad_kernel<D, BN, NSLOT, true> : sparse_attention_quad_kernel<D, BN, NSLOT, false>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES) != cudaSuccess)
+    return EI_ERR_CUDA;
+  kern<<<(unsigned)grid, QUAD_THREADS, L::DYN_BYTES, st>>>(tmq, tmk, tmv, a.out, a.items, a.indices, a.status, s, scale_log2,
+                                                          a.skip_log2, pk, npk);
+  return cudaGetLastError() == cudaSuccess ? EI_OK : EI_ERR_CUDA;
+}
+
 int launch_attention_quad(const Shape& s, const AttnArgs& a, cudaStream_t st) {
   constexpr int D = 128, BN = 128, NSLOT = 5;
   using L = QuadSmem<D, BN, NSLOT>;
@@ -1182,7 +1219,7 @@ int launch_attention_quad(const Shape& s, const AttnArgs& a, cudaStream_t st) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES) != cudaSuccess)
       return EI_ERR_CUDA;
     kern<<<(unsigned)n_items, QUAD_THREADS, L::DYN_BYTES, st>>>(tmq, tmk, tmv, a.out, a.items, a.indices, a.status, s,
-                                                               scale_log2, a.skip_log2);
+                                                               scale_log2, a.skip_log2, nullptr, 0);
   }
   return cudaGetLastError() == cudaSuccess ? EI_OK : EI_ERR_CUDA;
 }

@@ -33,6 +33,37 @@ __host__ __device__ inline int causal_blocks(const Shape& s, int i) {
   return c < s.C_B ? c : s.C_B;
 }
 
+// One sequence of a packed batch that runs in ONE set of launches (ei_prefill_varlen): its shape and where its
+// share of every plan table starts.  A planning / attention kernel that is handed such a table looks its CTA's
+// sequence up (w_* = CTAs of the earlier sequences in that kernel's grid) and then works on the sequence as if it
+// were alone: the tables of the sequences lie one after another, each laid out exactly as a plan of that
+// sequence would lay them out.
+struct PackedSeq {
+  Shape s;
+  long long tok0;   // first token of the sequence in q, k, v, out
+  long long cell0;  // first (head, segment) cell: entropy, multipliers, counts, query representatives, stage-4 records
+  long long off0;   // first entry of its offsets (cells + 1 entries per sequence)
+  long long sc0;    // first score
+  long long kb0;    // first key block in the K-representative arrays (KV-head stride there: the sequence's own C_B)
+  long long idx0;   // first list entry
+  long long T;      // TOTAL mode: the sequence's total
+  int head0;        // first class entry
+  int index;        // position among the sequences of this set of launches (its Stats slot)
+  int w_pool, w_obs, w_sel, w_att;
+};
+constexpr int MAX_PACKED = 256;  // sequences per set of launches
+#ifdef __CUDACC__
+__device__ __forceinline__ int packed_find(const PackedSeq* pk, int npk, int bid, int PackedSeq::*w) {
+  int lo = 0, hi = npk;  // the last sequence whose first CTA is <= bid
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (pk[mid].*w <= bid) lo = mid;
+    else hi = mid;
+  }
+  return lo;
+}
+#endif
+
 struct Stats {  // EI_ITEM_STATS
   long long total, rigid_heads, b_star, leftover, min_k, max_k, pv_skipped, reserved1;  // pv_skipped: counted by stage 4
 };
@@ -41,6 +72,20 @@ struct Stats {  // EI_ITEM_STATS
 int shape_from_params(const ei_params* p, Shape* s);
 
 // ---- launch wrappers (each returns a cudaError_t from the launch) -----------------------------
+// The *_packed forms run one launch over all npk sequences of pk (device array; pk_host the same on the host,
+// for the grid sizes); the table pointers are the plan's, the per-sequence offsets come from pk.
+cudaError_t launch_pool_packed(const PackedSeq* pk, const PackedSeq* pk_host, int npk, const __nv_bfloat16* q,
+                               const __nv_bfloat16* k, __nv_bfloat16* qmax, __nv_bfloat16* qmin, __nv_bfloat16* kmax,
+                               __nv_bfloat16* kmin, cudaStream_t st);
+cudaError_t launch_observe_packed(const PackedSeq* pk, const PackedSeq* pk_host, int npk, const __nv_bfloat16* qmax,
+                                  const __nv_bfloat16* qmin, const __nv_bfloat16* kmax, const __nv_bfloat16* kmin,
+                                  double scale, float* scores, float* entropy, cudaStream_t st);
+struct BudgetArgs;
+void packed_fill_work(PackedSeq* pk_host, int npk);  // fills w_pool, w_obs, w_sel, w_att
+cudaError_t launch_budget_packed(const PackedSeq* pk, int npk, const BudgetArgs& a, const float* entropy,
+                                 unsigned char* rigid, int* Mfx, int* kblocks, int* offsets, Stats* stats, cudaStream_t st);
+cudaError_t launch_select_packed(const PackedSeq* pk, const PackedSeq* pk_host, int npk, const float* scores,
+                                 const int* kblocks, const int* offsets, int* indices, int* items, cudaStream_t st);
 cudaError_t launch_pool(const Shape& s, const __nv_bfloat16* q, const __nv_bfloat16* k,
                         __nv_bfloat16* qmax, __nv_bfloat16* qmin, __nv_bfloat16* kmax,
                         __nv_bfloat16* kmin, int first_block, cudaStream_t st);
@@ -56,6 +101,7 @@ cudaError_t launch_observe(const Shape& s, const __nv_bfloat16* qmax, const __nv
                            const __nv_bfloat16* kmax, const __nv_bfloat16* kmin, double scale,
                            float* scores, float* entropy, cudaStream_t st);
 bool observe_shape_supported(const Shape& s);
+int observe_ctas_per_row(const Shape& s);  // CTAs per (KV head, segment) row of the observation kernel's grid
 
 // K blocks only (the query cells are then pooled by the fused kernel below)
 cudaError_t launch_pool_k(const Shape& s, const __nv_bfloat16* k, __nv_bfloat16* kmax, __nv_bfloat16* kmin,
@@ -113,6 +159,10 @@ struct AttnArgs {
 int launch_attention(const Shape& s, const AttnArgs& a, cudaStream_t st);
 int launch_attention_quad(const Shape& s, const AttnArgs& a, cudaStream_t st);  // d = 128, L_B = 128, L_S % 256 = 0
 int launch_attention_tri(const Shape& s, const AttnArgs& a, cudaStream_t st);   // same shapes
+// the per-CTA quad-layout kernel over all sequences of a packed batch (a.q .. a.out: the packed tensors, a.items /
+// a.indices: the plan's arrays; offsets and shapes per sequence from pk)
+int launch_attention_quad_packed(const PackedSeq* pk, const PackedSeq* pk_host, int npk, long long n_tokens,
+                                 const AttnArgs& a, cudaStream_t st);
 // one record of 8 ints per (list cell, tile pair) from the plan's lists (ls: the list-head shape); a no-op for
 // shapes the tile-pair kernels do not take
 cudaError_t launch_attention_items(const Shape& ls, const int* offsets, const int* indices, int* items, cudaStream_t st);

@@ -49,7 +49,7 @@ __global__ void __launch_bounds__(256) pool_kernel(const __nv_bfloat16* __restri
                                                    __nv_bfloat16* __restrict__ qmin,
                                                    __nv_bfloat16* __restrict__ kmax,
                                                    __nv_bfloat16* __restrict__ kmin, Shape s, long long cell0,
-                                                   int kb0) {
+                                                   int kb0, const PackedSeq* pk, int npk) {
   constexpr int LPR = D / 8;     // 16-byte lanes per row
   constexpr int RS = 256 / LPR;  // rows per pass
   constexpr int UNROLL = 8;
@@ -58,7 +58,19 @@ __global__ void __launch_bounds__(256) pool_kernel(const __nv_bfloat16* __restri
 
   const int tid = threadIdx.x;
   const int lane16 = tid % LPR, slot = tid / LPR;
-  long long cell = cell0 + blockIdx.x;  // cell0 = s.cells pools the K blocks only
+  int bid = blockIdx.x;
+  if (pk != nullptr) {  // a packed batch: my sequence's shape, my CTA's number within it, its share of the tables
+    const PackedSeq& P = pk[packed_find(pk, npk, bid, &PackedSeq::w_pool)];
+    s = P.s;
+    bid -= P.w_pool;
+    q += P.tok0 * s.qs_t;
+    k += P.tok0 * s.ks_t;
+    qmax += P.cell0 * D;
+    qmin += P.cell0 * D;
+    kmax += P.kb0 * D;
+    kmin += P.kb0 * D;
+  }
+  long long cell = cell0 + bid;  // cell0 = s.cells pools the K blocks only
   const __nv_bfloat16* base;
   long long tok_stride;
   int L;
@@ -126,11 +138,25 @@ cudaError_t launch_pool(const Shape& s, const __nv_bfloat16* q, const __nv_bfloa
                         __nv_bfloat16* kmin, int first_block, cudaStream_t st) {
   const long long grid = s.cells + (long long)s.Hkv * max(0, s.C_B - first_block);
   if (s.d == 256)
-    pool_kernel<256><<<(unsigned)grid, 256, 0, st>>>(q, k, qmax, qmin, kmax, kmin, s, 0, first_block);
+    pool_kernel<256><<<(unsigned)grid, 256, 0, st>>>(q, k, qmax, qmin, kmax, kmin, s, 0, first_block, nullptr, 0);
   else if (s.d == 128)
-    pool_kernel<128><<<(unsigned)grid, 256, 0, st>>>(q, k, qmax, qmin, kmax, kmin, s, 0, first_block);
+    pool_kernel<128><<<(unsigned)grid, 256, 0, st>>>(q, k, qmax, qmin, kmax, kmin, s, 0, first_block, nullptr, 0);
   else
-    pool_kernel<64><<<(unsigned)grid, 256, 0, st>>>(q, k, qmax, qmin, kmax, kmin, s, 0, first_block);
+    pool_kernel<64><<<(unsigned)grid, 256, 0, st>>>(q, k, qmax, qmin, kmax, kmin, s, 0, first_block, nullptr, 0);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_pool_packed(const PackedSeq* pk, const PackedSeq* pk_host, int npk, const __nv_bfloat16* q,
+                               const __nv_bfloat16* k, __nv_bfloat16* qmax, __nv_bfloat16* qmin, __nv_bfloat16* kmax,
+                               __nv_bfloat16* kmin, cudaStream_t st) {
+  const Shape& s = pk_host[npk - 1].s;
+  const long long grid = pk_host[npk - 1].w_pool + s.cells + (long long)s.Hkv * s.C_B;
+  if (s.d == 256)
+    pool_kernel<256><<<(unsigned)grid, 256, 0, st>>>(q, k, qmax, qmin, kmax, kmin, s, 0, 0, pk, npk);
+  else if (s.d == 128)
+    pool_kernel<128><<<(unsigned)grid, 256, 0, st>>>(q, k, qmax, qmin, kmax, kmin, s, 0, 0, pk, npk);
+  else
+    pool_kernel<64><<<(unsigned)grid, 256, 0, st>>>(q, k, qmax, qmin, kmax, kmin, s, 0, 0, pk, npk);
   return cudaGetLastError();
 }
 
@@ -139,11 +165,11 @@ cudaError_t launch_pool_k(const Shape& s, const __nv_bfloat16* k, __nv_bfloat16*
   const long long grid = (long long)s.Hkv * (s.C_B - first_block);
   if (grid <= 0) return cudaSuccess;
   if (s.d == 256)
-    pool_kernel<256><<<(unsigned)grid, 256, 0, st>>>(nullptr, k, nullptr, nullptr, kmax, kmin, s, s.cells, first_block);
+    pool_kernel<256><<<(unsigned)grid, 256, 0, st>>>(nullptr, k, nullptr, nullptr, kmax, kmin, s, s.cells, first_block, nullptr, 0);
   else if (s.d == 128)
-    pool_kernel<128><<<(unsigned)grid, 256, 0, st>>>(nullptr, k, nullptr, nullptr, kmax, kmin, s, s.cells, first_block);
+    pool_kernel<128><<<(unsigned)grid, 256, 0, st>>>(nullptr, k, nullptr, nullptr, kmax, kmin, s, s.cells, first_block, nullptr, 0);
   else
-    pool_kernel<64><<<(unsigned)grid, 256, 0, st>>>(nullptr, k, nullptr, nullptr, kmax, kmin, s, s.cells, first_block);
+    pool_kernel<64><<<(unsigned)grid, 256, 0, st>>>(nullptr, k, nullptr, nullptr, kmax, kmin, s, s.cells, first_block, nullptr, 0);
   return cudaGetLastError();
 }
 
@@ -199,7 +225,7 @@ __global__ void __launch_bounds__(OBS_THREADS, 1)
 observe_kernel(const __nv_bfloat16* __restrict__ qmax, const __nv_bfloat16* __restrict__ qmin,
                const __nv_bfloat16* __restrict__ kmax, const __nv_bfloat16* __restrict__ kmin,
                float* __restrict__ scores, float* __restrict__ entropy, Shape s, double scale,
-               int nsub, int xcap) {
+               int nsub, int xcap, const PackedSeq* pk, int npk) {
   extern __shared__ __align__(16) unsigned char obs_smem[];
   // layout: lse [HG*4] double | epart [HG][OBS_WARPS] double | xs [HG*4][xcap] double
   double* lse = reinterpret_cast<double*>(obs_smem);
@@ -209,6 +235,17 @@ observe_kernel(const __nv_bfloat16* __restrict__ qmax, const __nv_bfloat16* __re
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   // longest rows first
   int bid = blockIdx.x;
+  if (pk != nullptr) {  // a packed batch: my sequence's shape, my CTA's number within it, its share of the tables
+    const PackedSeq& P = pk[packed_find(pk, npk, bid, &PackedSeq::w_obs)];
+    s = P.s;
+    bid -= P.w_obs;
+    qmax += P.cell0 * D;
+    qmin += P.cell0 * D;
+    kmax += P.kb0 * D;
+    kmin += P.kb0 * D;
+    scores += P.sc0;
+    entropy += P.cell0;
+  }
   const int sub = bid % nsub;
   bid /= nsub;
   const int g = bid % s.Hkv;
@@ -356,21 +393,53 @@ bool observe_shape_supported(const Shape& s) { return observe_pick_hg(s) != 0; }
 template <int D, int HG>
 static cudaError_t launch_observe_t(const Shape& s, const __nv_bfloat16* qmax, const __nv_bfloat16* qmin,
                                     const __nv_bfloat16* kmax, const __nv_bfloat16* kmin, double scale,
-                                    float* scores, float* entropy, cudaStream_t st) {
+                                    float* scores, float* entropy, cudaStream_t st, const PackedSeq* pk = nullptr,
+                                    int npk = 0, long long packed_grid = 0) {
+  // (packed: s is the sequence with the most key blocks -- it sizes the shared-memory staging -- and the grid
+  //  covers all sequences, w_obs counting C_S * H_kv * nsub CTAs per sequence)
   const int nsub = (s.G + HG - 1) / HG;
   const size_t smem = observe_smem_bytes(D, HG, s.C_B);
   cudaError_t e = cudaFuncSetAttribute(observe_kernel<D, HG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  const unsigned grid = (unsigned)((long long)s.C_S * s.Hkv * nsub);
-  observe_kernel<D, HG><<<grid, OBS_THREADS, smem, st>>>(qmax, qmin, kmax, kmin, scores, entropy, s, scale, nsub, s.C_B);
+  const unsigned grid = (unsigned)(pk ? packed_grid * nsub : (long long)s.C_S * s.Hkv * nsub);
+  observe_kernel<D, HG><<<grid, OBS_THREADS, smem, st>>>(qmax, qmin, kmax, kmin, scores, entropy, s, scale, nsub, s.C_B,
+                                                         pk, npk);
   return cudaGetLastError();
 }
+
+int observe_ctas_per_row(const Shape& s) {  // CTAs per (KV head, segment) row: the head sub-groups
+  const int hg = observe_pick_hg(s);
+  return hg ? (s.G + hg - 1) / hg : 0;
+}
+
+static cudaError_t launch_observe_any(const Shape& s, const __nv_bfloat16* qmax, const __nv_bfloat16* qmin,
+                                      const __nv_bfloat16* kmax, const __nv_bfloat16* kmin, double scale, float* scores,
+                                      float* entropy, cudaStream_t st, const PackedSeq* pk, int npk, long long packed_rows);
 
 cudaError_t launch_observe(const Shape& s, const __nv_bfloat16* qmax, const __nv_bfloat16* qmin,
                            const __nv_bfloat16* kmax, const __nv_bfloat16* kmin, double scale,
                            float* scores, float* entropy, cudaStream_t st) {
+  return launch_observe_any(s, qmax, qmin, kmax, kmin, scale, scores, entropy, st, nullptr, 0, 0);
+}
+
+// pk_host[i].w_obs counts (KV head, segment) ROWS of the earlier sequences times the CTAs per row
+cudaError_t launch_observe_packed(const PackedSeq* pk, const PackedSeq* pk_host, int npk, const __nv_bfloat16* qmax,
+                                  const __nv_bfloat16* qmin, const __nv_bfloat16* kmax, const __nv_bfloat16* kmin,
+                                  double scale, float* scores, float* entropy, cudaStream_t st) {
+  int big = 0;
+  long long rows = 0;
+  for (int i = 0; i < npk; ++i) {
+    if (pk_host[i].s.C_B > pk_host[big].s.C_B) big = i;
+    rows += (long long)pk_host[i].s.C_S * pk_host[i].s.Hkv;
+  }
+  return launch_observe_any(pk_host[big].s, qmax, qmin, kmax, kmin, scale, scores, entropy, st, pk, npk, rows);
+}
+
+static cudaError_t launch_observe_any(const Shape& s, const __nv_bfloat16* qmax, const __nv_bfloat16* qmin,
+                                      const __nv_bfloat16* kmax, const __nv_bfloat16* kmin, double scale, float* scores,
+                                      float* entropy, cudaStream_t st, const PackedSeq* pk, int npk, long long packed_rows) {
   const int hg = observe_pick_hg(s);
-#define EI_OBS(D_, HG_) return launch_observe_t<D_, HG_>(s, qmax, qmin, kmax, kmin, scale, scores, entropy, st)
+#define EI_OBS(D_, HG_) return launch_observe_t<D_, HG_>(s, qmax, qmin, kmax, kmin, scale, scores, entropy, st, pk, npk, packed_rows)
   if (s.d == 256) {
     if (hg == 4) EI_OBS(256, 4);
     if (hg == 2) EI_OBS(256, 2);
@@ -811,7 +880,19 @@ __device__ long long block_excl_scan(long long v, long long* warp_sums, long lon
 __global__ void __launch_bounds__(BUD_THREADS, 1)
 budget_kernel(Shape s, BudgetArgs a, const float* __restrict__ entropy, unsigned char* __restrict__ rigid,
               int* __restrict__ Mfx, const int* Mall, int* __restrict__ kblocks, int* __restrict__ offsets,
-              Stats* __restrict__ stats) {
+              Stats* __restrict__ stats, const PackedSeq* pk) {
+  if (pk != nullptr) {  // a packed batch: one CTA per sequence, each on its own share of the tables
+    const PackedSeq& P = pk[blockIdx.x];
+    s = P.s;
+    a.T = P.T;
+    a.H_all = s.H;
+    entropy += P.cell0;
+    rigid += P.head0;
+    Mfx += P.cell0;
+    kblocks += P.cell0;
+    offsets += P.off0;
+    stats += P.index;
+  }
   __shared__ long long s_warp[33];
   __shared__ int s_rigid, s_mink, s_maxk;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -994,7 +1075,13 @@ budget_kernel(Shape s, BudgetArgs a, const float* __restrict__ entropy, unsigned
 
 cudaError_t launch_budget(const Shape& s, const BudgetArgs& a, const float* entropy, unsigned char* rigid,
                           int* Mfx, const int* Mall, int* kblocks, int* offsets, Stats* stats, cudaStream_t st) {
-  budget_kernel<<<1, BUD_THREADS, 0, st>>>(s, a, entropy, rigid, Mfx, Mall, kblocks, offsets, stats);
+  budget_kernel<<<1, BUD_THREADS, 0, st>>>(s, a, entropy, rigid, Mfx, Mall, kblocks, offsets, stats, nullptr);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_budget_packed(const PackedSeq* pk, int npk, const BudgetArgs& a, const float* entropy,
+                                 unsigned char* rigid, int* Mfx, int* kblocks, int* offsets, Stats* stats, cudaStream_t st) {
+  budget_kernel<<<npk, BUD_THREADS, 0, st>>>(Shape{}, a, entropy, rigid, Mfx, nullptr, kblocks, offsets, stats, pk);
   return cudaGetLastError();
 }
 
@@ -1016,10 +1103,22 @@ __device__ __forceinline__ uint32_t order_key(float f) {
 
 __global__ void __launch_bounds__(SEL_WARPS * 32)
 select_kernel(Shape s, const float* __restrict__ scores, const int* __restrict__ kblocks,
-              const int* __restrict__ offsets, int* __restrict__ indices, int* __restrict__ items, int pairs_per_seg) {
+              const int* __restrict__ offsets, int* __restrict__ indices, int* __restrict__ items, int pairs_per_seg,
+              const PackedSeq* pk, int npk) {
   __shared__ int hist[SEL_WARPS][256];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const long long c = (long long)blockIdx.x * SEL_WARPS + warp;
+  int bid = blockIdx.x;
+  if (pk != nullptr) {  // a packed batch: my sequence's shape, my CTA's number within it, its share of the tables
+    const PackedSeq& P = pk[packed_find(pk, npk, bid, &PackedSeq::w_sel)];
+    s = P.s;
+    bid -= P.w_sel;
+    scores += P.sc0;
+    kblocks += P.cell0;
+    offsets += P.off0;
+    indices += P.idx0;
+    if (items != nullptr) items += P.cell0 * pairs_per_seg * 8;
+  }
+  const long long c = (long long)bid * SEL_WARPS + warp;
   if (c >= s.cells) return;
   const int h = (int)(c / s.C_S), i = (int)(c % s.C_S);
   const float* row = scores + (long long)h * s.SC + row_offset(s, i);
@@ -1113,7 +1212,37 @@ cudaError_t launch_select(const Shape& s, const float* scores, const int* kblock
                           int* indices, int* items, cudaStream_t st) {
   const unsigned grid = (unsigned)((s.cells + SEL_WARPS - 1) / SEL_WARPS);
   const int pairs = s.L_S % 256 == 0 ? s.L_S / 256 : 0;  // shapes the tile-pair kernels of stage 4 take
-  select_kernel<<<grid, SEL_WARPS * 32, 0, st>>>(s, scores, kblocks, offsets, indices, pairs ? items : nullptr, pairs);
+  select_kernel<<<grid, SEL_WARPS * 32, 0, st>>>(s, scores, kblocks, offsets, indices, pairs ? items : nullptr, pairs,
+                                                 nullptr, 0);
+  return cudaGetLastError();
+}
+
+// grid bookkeeping of a packed batch: CTAs of the earlier sequences in each kernel's grid
+void packed_fill_work(PackedSeq* pk_host, int npk) {
+  int big = 0;
+  for (int i = 0; i < npk; ++i)
+    if (pk_host[i].s.C_B > pk_host[big].s.C_B) big = i;
+  const int nsub = observe_ctas_per_row(pk_host[big].s);
+  long long wp = 0, wo = 0, ws = 0, wa = 0;
+  for (int i = 0; i < npk; ++i) {
+    const Shape& s = pk_host[i].s;
+    pk_host[i].w_pool = (int)wp;
+    pk_host[i].w_obs = (int)wo;
+    pk_host[i].w_sel = (int)ws;
+    pk_host[i].w_att = (int)wa;
+    wp += s.cells + (long long)s.Hkv * s.C_B;
+    wo += (long long)s.C_S * s.Hkv * nsub;
+    ws += (s.cells + SEL_WARPS - 1) / SEL_WARPS;
+    wa += (long long)s.H * s.C_S * (s.L_S / 256);
+  }
+}
+
+cudaError_t launch_select_packed(const PackedSeq* pk, const PackedSeq* pk_host, int npk, const float* scores,
+                                 const int* kblocks, const int* offsets, int* indices, int* items, cudaStream_t st) {
+  const Shape& s = pk_host[npk - 1].s;
+  const unsigned grid = (unsigned)(pk_host[npk - 1].w_sel + (s.cells + SEL_WARPS - 1) / SEL_WARPS);
+  const int pairs = s.L_S % 256 == 0 ? s.L_S / 256 : 0;
+  select_kernel<<<grid, SEL_WARPS * 32, 0, st>>>(s, scores, kblocks, offsets, indices, pairs ? items : nullptr, pairs, pk, npk);
   return cudaGetLastError();
 }
 

@@ -105,3 +105,56 @@ def test_packed_batch_arguments_are_checked():
     assert not out.any()                                             # nothing was launched
     pl.prefill_varlen(qd, kd, vd, out, [0, 0])                       # an empty batch is fine
     assert pl.status() == 0
+
+
+@pytest.mark.parametrize("mode", ["total", "base"])
+@pytest.mark.parametrize("layout", ["head_major", "token_major"])
+def test_packed_batch_in_one_set_of_launches(mode, layout):
+    # A plan made for the batch's total length has room for every sequence's tables side by side: the whole batch
+    # then costs five launches (pool, observe, budget, select, attention), however many sequences it has -- and
+    # still equals per-sequence calls bit for bit.
+    rng = np.random.default_rng(7)
+    if mode == "base":
+        lens = [int(x) for x in rng.integers(130, 2100, size=11)] + [0, 2048, 129]
+    else:                                               # long enough that half the causal blocks cover the diagonal ones
+        lens = [int(x) for x in rng.integers(1700, 3000, size=8)] + [0, 2048, 1701]
+    total = sum(lens)
+    q, k, v, (qd, kd, vd) = packed(layout, lens, seed=151)
+    fraction, base = (0.5, None) if mode == "total" else (0.0, 640.0)
+    # (room for every sequence's segments: each sequence rounds up to whole segments of its own)
+    p = ei.params_default(H, HKV, D, sum(-(-n // L_S) * L_S for n in lens), L_S, L_B, fraction)
+    if base is not None:
+        p.base_budget_tokens = base
+    if layout == "token_major":
+        p.q_stride_tok = p.o_stride_tok = H * D
+        p.k_stride_tok = p.v_stride_tok = HKV * D
+        p.q_stride_head = p.k_stride_head = p.v_stride_head = p.o_stride_head = D
+    else:
+        p.q_stride_head = p.k_stride_head = p.v_stride_head = p.o_stride_head = total * D
+    pl = ei.Plan(p)
+    out = torch.full(qd.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    n0 = pl.launches()
+    pl.prefill_varlen(qd, kd, vd, out, cu)
+    assert pl.status() == 0
+    assert pl.launches() - n0 == 5
+    got = to_bits(out)
+    if layout == "token_major":
+        got = np.ascontiguousarray(got.reshape(total, H, D).transpose(1, 0, 2))
+    got = got.reshape(H, total, D)
+    for b, n in enumerate(lens):
+        if n == 0:
+            continue
+        lo, hi = int(cu[b]), int(cu[b + 1])
+        qs, ks, vs = (np.ascontiguousarray(a[:, lo:hi]) for a in (q, k, v))
+        p1 = ei.params_default(H, HKV, D, n, L_S, L_B, fraction)
+        if base is not None:
+            p1.base_budget_tokens = base
+        ref = ei.Plan(p1)
+        o1 = torch.empty((H, n, D), dtype=torch.bfloat16, device="cuda")
+        ref.plan(to_dev(qs), to_dev(ks))
+        ref.sparse_prefill(to_dev(qs), to_dev(ks), to_dev(vs), o1)
+        np.testing.assert_array_equal(got[:, lo:hi], to_bits(o1).reshape(H, n, D), err_msg=f"sequence {b} of {n} tokens")
+    with pytest.raises(ei.EiError) as e:                # the tables hold a batch now: nothing to attend from
+        pl.sparse_prefill(qd, kd, vd, out)
+    assert e.value.code == ei.STATUS["NOT_PLANNED"]
