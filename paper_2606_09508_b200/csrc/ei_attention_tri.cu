@@ -120,15 +120,15 @@ __device__ __forceinline__ bool softmax_block(uint32_t t_s, uint32_t t_o, uint32
   uint32_t xa[32], xb[32];  // columns 0..63 and 64..127: [4i + {0,1}] row A, [4i + {2,3}] row B, columns 8i + 2*(lane%4) + {0,1}
   ld_16x64(t_s, xa);
   ld_16x64(t_s + 64, xb);
-  // while the logits are on their way: the reference valid after block J - 1, from the warp of the other set that
-  // owns my rows
+  tmem_wait_ld();  // (nothing that may call a function between the loads and this wait: the loads land in the
+                   //  registers asynchronously, and a call could save and restore them in between)
+  // the reference valid after block J - 1, from the warp of the other set that owns my rows
   float pmA = 0.f, pmB = 0.f;
   if (!first) {
     ok = mbar_wait(bar_mx_other, par_mx_other, status) && ok;
     pmA = mref_other[lane >> 2];
     pmB = mref_other[(lane >> 2) + 8];
   }
-  tmem_wait_ld();
   if (masked) {
 #pragma unroll
     for (int ii = 0; ii < 8; ++ii) {
