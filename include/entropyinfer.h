@@ -249,10 +249,11 @@ int ei_plan_pooled(ei_plan_t* plan, void* stream);
    entries: a plan created for the batch's total length, each sequence rounded up to whole segments, holds them
    all; at most 256 at a time) run in ONE set of five launches -- pooling, observation, budget (one CTA per
    sequence), selection, attention -- in which every CTA looks up its sequence in a small table copied to the
-   device with the call; this applies to head_dim 128, block_len 128, segments a multiple of 256, per-head lists
-   and the default attention kernel.  A sequence that fits only on its own (a plan made for the longest sequence),
-   and every sequence under group-shared lists, the other kernels or other shapes, takes the plan re-targeted to
-   it and the ordinary two calls (four to five launches per sequence).  The results are the same either way.
+   device with the call (group-shared lists: a sixth launch for the aggregation); this applies to every shape
+   with the attention kernel the library picks by default.  A sequence that fits only on its own (a plan made
+   for the longest sequence), and every sequence of a plan whose flags name another attention kernel, takes the
+   plan re-targeted to it and the ordinary two calls (four to five launches per sequence).  The results are the
+   same either way.
    Asynchronous; afterwards the plan is targeted at the last non-empty sequence.  It holds that sequence's
    tables when the sequence ran on its own; after a set of packed launches the tables hold the batch, one
    sequence after another, and ei_sparse_prefill returns EI_ERR_NOT_PLANNED until the next ei_plan.          */

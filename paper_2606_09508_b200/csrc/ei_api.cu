@@ -742,15 +742,13 @@ int ei_plan_set_lengths(ei_plan_t* pl, int seq_len, int q_len, int k_blocks_vali
 }
 
 namespace {
-// Can a packed batch run in one set of launches on this plan?  (The staged planning kernels and the default
-// stage-4 kernel take the per-sequence table; group-shared lists, the other attention kernels and the other
-// shapes go sequence by sequence.)
+// Can a packed batch run in one set of launches on this plan?  (The staged planning kernels and the stage-4
+// kernels picked by default take the per-sequence table; the kernels behind flags go sequence by sequence.)
 bool packed_capable(const ei_plan_t* pl) {
-  const ei::Shape& s = pl->shape;
-  const uint32_t other = EI_FLAG_GROUP_SHARED | EI_FLAG_ATTN_SPLIT | EI_FLAG_ATTN_SKIP_ZERO_PV | EI_FLAG_ATTN_P_VIA_SMEM |
+  const uint32_t other = EI_FLAG_ATTN_SPLIT | EI_FLAG_ATTN_SKIP_ZERO_PV | EI_FLAG_ATTN_P_VIA_SMEM |
                          EI_FLAG_ATTN_PAIR_8WARP | EI_FLAG_ATTN_PERSISTENT | EI_FLAG_ATTN_SINGLE_TILE | EI_FLAG_ATTN_TRI |
                          EI_FLAG_ATTN_QUAD;
-  return s.L_S % 256 == 0 && s.d == 128 && s.L_B == 128 && !(pl->params.flags & other);
+  return !(pl->params.flags & other);
 }
 
 // sequences [b0, b1) of the batch (all non-empty, all fitting the plan's tables together) in five launches
@@ -777,10 +775,16 @@ int run_packed(ei_plan_t* pl, const std::vector<ei::PackedSeq>& seqs_in, long lo
   a.phase = ei::EI_BUDGET_PHASE_ALL;
   a.H_all = 0;
   a.first_head = 0;
+  if (e == cudaSuccess && pl->group) {
+    e = ei::launch_group_aggregate_packed(pl->pk, hp.data(), n, pl->scores, pl->entropy, pl->g_scores, pl->g_entropy, st);
+    pl->launches += 1;
+  }
   if (e == cudaSuccess)
-    e = ei::launch_budget_packed(pl->pk, n, a, pl->entropy, pl->rigid, pl->Mfx, pl->kblocks, pl->offsets, pl->stats, st);
+    e = ei::launch_budget_packed(pl->pk, n, a, pl->group ? pl->g_entropy : pl->entropy, pl->rigid, pl->Mfx, pl->kblocks,
+                                 pl->offsets, pl->stats, st);
   if (e == cudaSuccess)
-    e = ei::launch_select_packed(pl->pk, hp.data(), n, pl->scores, pl->kblocks, pl->offsets, pl->indices, pl->items, st);
+    e = ei::launch_select_packed(pl->pk, hp.data(), n, pl->group ? pl->g_scores : pl->scores, pl->kblocks, pl->offsets,
+                                 pl->indices, pl->items, st);
   pl->launches += 4;
   if (e != cudaSuccess) return EI_ERR_CUDA;
   ei::AttnArgs at{};
@@ -794,7 +798,7 @@ int run_packed(ei_plan_t* pl, const std::vector<ei::PackedSeq>& seqs_in, long lo
   at.status = pl->status;
   at.scale = (float)pl->attn_scale;
   at.skip_log2 = (pl->params.flags & EI_FLAG_ATTN_NO_SKIP) ? INFINITY : 24.0f;
-  const int rc = ei::launch_attention_quad_packed(pl->pk, hp.data(), n, n_tokens, at, st);
+  const int rc = ei::launch_attention_packed(pl->pk, hp.data(), n, n_tokens, at, st);
   pl->launches += 1;
   return rc;
 }
@@ -825,6 +829,8 @@ int ei_prefill_varlen(ei_plan_t* pl, const void* q, const void* k, const void* v
     ei::PackedSeq P{};
     P.s = pl->shape;
     P.s.KB_cap = P.s.C_B;  // its K representatives are laid out as a plan of this sequence alone would lay them out
+    P.ls = pl->lshape;
+    P.ls.KB_cap = P.ls.C_B;
     P.tok0 = cu[b];
     P.T = pl->T;
     P.index = b;  // (the batch position for now; the slot within its set of launches is assigned below)
@@ -841,23 +847,28 @@ int ei_prefill_varlen(ei_plan_t* pl, const void* q, const void* k, const void* v
   while (i0 < seqs.size()) {
     // the longest run of sequences from i0 on whose tables fit the plan's side by side
     size_t i1 = i0;
-    long long cells = 0, sc = 0, kb = 0, idx = 0;
+    long long cells = 0, sc = 0, kb = 0, idx = 0, lcells = 0, lsc = 0;
     std::vector<ei::PackedSeq> grp;
     while (packed_ok && i1 < seqs.size() && (int)grp.size() < ei::MAX_PACKED) {
-      const ei::Shape& sb = seqs[i1].s;
+      const ei::Shape &sb = seqs[i1].s, &lb = seqs[i1].ls;
       if (cells + sb.cells > pl->cap_cells || sc + (long long)sb.H * sb.SC > pl->cap_scores ||
+          lcells + lb.cells > pl->cap_lcells || lsc + (long long)lb.H * lb.SC > pl->cap_lscores ||
           kb + (long long)sb.Hkv * sb.C_B > kreps_cap || idx + need[i1] > pl->capacity)
         break;
       ei::PackedSeq P = seqs[i1];
       P.cell0 = cells;
-      P.off0 = cells + (long long)grp.size();
+      P.lcell0 = lcells;
+      P.off0 = lcells + (long long)grp.size();
       P.sc0 = sc;
+      P.lsc0 = lsc;
       P.kb0 = kb;
       P.idx0 = idx;
-      P.head0 = (int)grp.size() * sb.H;
+      P.head0 = (int)grp.size() * lb.H;
       P.index = (int)grp.size();
       grp.push_back(P);
       cells += sb.cells;
+      lcells += lb.cells;
+      lsc += (long long)lb.H * lb.SC;
       sc += (long long)sb.H * sb.SC;
       kb += (long long)sb.Hkv * sb.C_B;
       idx += need[i1];

@@ -53,7 +53,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 1)
 sparse_attention_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
                         const __grid_constant__ CUtensorMap tmv, __nv_bfloat16* __restrict__ out,
                         const int* __restrict__ offsets, const int* __restrict__ indices,
-                        int* __restrict__ status, Shape s, float scale_log2) {
+                        int* __restrict__ status, Shape s, float scale_log2, const PackedSeq* pk, int npk) {
   using L = AttSmem<D, BN, NS, P_SMEM>;
   extern __shared__ unsigned char att_smem_raw[];
 
@@ -73,6 +73,16 @@ sparse_attention_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_co
   // ---- which tile ---------------------------------------------------------------------------------
   const int tiles_per_seg = s.L_S / BM;
   int bid = blockIdx.x;
+  int tok0 = 0;  // a packed batch: my sequence starts here in q, k, v, out (the tensor maps span the whole batch)
+  if (pk != nullptr) {
+    const PackedSeq& P = pk[packed_find(pk, npk, bid, &PackedSeq::w_att)];
+    s = P.s;
+    bid -= P.w_att;
+    tok0 = (int)P.tok0;
+    offsets += P.off0;
+    indices += P.idx0;
+    out += P.tok0 * s.os_t;
+  }
   const int qt = bid % tiles_per_seg;
   bid /= tiles_per_seg;
   const int h = bid % s.H;
@@ -128,7 +138,7 @@ sparse_attention_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_co
     {
       mbar_expect_tx(BAR(B_QFULL), L::Q_BYTES);
 #pragma unroll
-      for (int p = 0; p < D / 64; ++p) tma_load_3d(sQ + p * (BM * 128), &tmq, p * 64, q0, h, BAR(B_QFULL));
+      for (int p = 0; p < D / 64; ++p) tma_load_3d(sQ + p * (BM * 128), &tmq, p * 64, tok0 + q0, h, BAR(B_QFULL));
       int issued = 0;
       for (int it = 0; it < n && ok; ++it) {
         const int st = it % NS;
@@ -139,7 +149,7 @@ sparse_attention_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_co
         mbar_expect_tx(BAR(B_KFULL + st), L::KV_BYTES);
 #pragma unroll
         for (int p = 0; p < D / 64; ++p)
-          tma_load_3d(sK + st * L::KV_BYTES + p * (BN * 128), &tmk, p * 64, blk * BN, g, BAR(B_KFULL + st));
+          tma_load_3d(sK + st * L::KV_BYTES + p * (BN * 128), &tmk, p * 64, tok0 + blk * BN, g, BAR(B_KFULL + st));
         ok = mbar_wait(BAR(B_VEMPTY + st), ph ^ 1, status);
         if (!ok) {  // the K load above is in flight: wait for it before leaving
           mbar_wait_drain(BAR(B_KFULL + st), ph);
@@ -148,7 +158,7 @@ sparse_attention_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_co
         mbar_expect_tx(BAR(B_VFULL + st), L::KV_BYTES);
 #pragma unroll
         for (int p = 0; p < D / 64; ++p)
-          tma_load_3d(sV + st * L::KV_BYTES + p * (BN * 128), &tmv, p * 64, blk * BN, g, BAR(B_VFULL + st));
+          tma_load_3d(sV + st * L::KV_BYTES + p * (BN * 128), &tmv, p * 64, tok0 + blk * BN, g, BAR(B_VFULL + st));
         issued = it + 1;
       }
       // Drain: every load this thread issued must have landed before the CTA's shared memory is released.
@@ -388,7 +398,7 @@ __global__ void __launch_bounds__(ATT2_THREADS, 1)
 sparse_attention_pair_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
                              const __grid_constant__ CUtensorMap tmv, __nv_bfloat16* __restrict__ out,
                              const int* __restrict__ offsets, const int* __restrict__ indices,
-                             int* __restrict__ status, Shape s, float scale_log2) {
+                             int* __restrict__ status, Shape s, float scale_log2, const PackedSeq* pk, int npk) {
   using L = Att2Smem<D, BN, NSLOT>;
   extern __shared__ unsigned char att_smem_raw[];
 
@@ -407,6 +417,16 @@ sparse_attention_pair_kernel(const __grid_constant__ CUtensorMap tmq, const __gr
 
   const int pairs_per_seg = s.L_S / (2 * BM);
   int bid = blockIdx.x;
+  int tok0 = 0;  // a packed batch: my sequence starts here in q, k, v, out (the tensor maps span the whole batch)
+  if (pk != nullptr) {
+    const PackedSeq& P = pk[packed_find(pk, npk, bid, &PackedSeq::w_att)];
+    s = P.s;
+    bid -= P.w_att;
+    tok0 = (int)P.tok0;
+    offsets += P.off0;
+    indices += P.idx0;
+    out += P.tok0 * s.os_t;
+  }
   const int pr = bid % pairs_per_seg;
   bid /= pairs_per_seg;
   const int h = bid % s.H;
@@ -466,7 +486,7 @@ sparse_attention_pair_kernel(const __grid_constant__ CUtensorMap tmq, const __gr
         mbar_expect_tx(BAR(B_QFULL + t), L::Q_BYTES);
 #pragma unroll
         for (int p = 0; p < D / 64; ++p)
-          tma_load_3d(sQ + t * L::Q_BYTES + p * (BM * 128), &tmq, p * 64, q0 + t * BM, h, BAR(B_QFULL + t));
+          tma_load_3d(sQ + t * L::Q_BYTES + p * (BM * 128), &tmq, p * 64, tok0 + q0 + t * BM, h, BAR(B_QFULL + t));
       }
       int issued = 0;  // ring items issued (K_j is item 2j, V_j is item 2j+1)
       for (int u = 0; u < 2 * n1; ++u) {
@@ -479,7 +499,7 @@ sparse_attention_pair_kernel(const __grid_constant__ CUtensorMap tmq, const __gr
         const CUtensorMap* tm = (u & 1) ? &tmv : &tmk;
 #pragma unroll
         for (int p = 0; p < D / 64; ++p)
-          tma_load_3d(sRing + slot * L::KV_BYTES + p * (BN * 128), tm, p * 64, blk * BN, g, BAR(B_FULL + slot));
+          tma_load_3d(sRing + slot * L::KV_BYTES + p * (BN * 128), tm, p * 64, tok0 + blk * BN, g, BAR(B_FULL + slot));
         issued = u + 1;
       }
       // Drain: every load issued here must have landed before the CTA's shared memory is released.
@@ -1669,41 +1689,45 @@ bool make_tensor_map(CUtensorMap* tm, const void* ptr, int d, int N, int heads, 
   return r == CUDA_SUCCESS;
 }
 
+// (pk != nullptr: one launch over the sequences of a packed batch -- the tensor maps then span the n_tokens rows of
+//  the packed tensors, `grid` counts the CTAs of all sequences and s is any one of them, for the strides)
 template <int D, int BN, int NS, bool P_SMEM>
-static int launch_t(const Shape& s, const AttnArgs& a, cudaStream_t st) {
+static int launch_t(const Shape& s, const AttnArgs& a, cudaStream_t st, const PackedSeq* pk = nullptr, int npk = 0,
+                    long long n_tokens = 0, long long packed_grid = 0) {
   using L = AttSmem<D, BN, NS, P_SMEM>;
   static_assert(L::DYN_BYTES <= 232448, "shared memory budget exceeded");
   CUtensorMap tmq, tmk, tmv;
-  if (!make_tensor_map(&tmq, a.q, D, s.Nq, s.H, s.qs_t, s.qs_h, BM) ||
-      !make_tensor_map(&tmk, a.k, D, s.N, s.Hkv, s.ks_t, s.ks_h, BN) ||
-      !make_tensor_map(&tmv, a.v, D, s.N, s.Hkv, s.vs_t, s.vs_h, BN))
+  if (!make_tensor_map(&tmq, a.q, D, pk ? (int)n_tokens : s.Nq, s.H, s.qs_t, s.qs_h, BM) ||
+      !make_tensor_map(&tmk, a.k, D, pk ? (int)n_tokens : s.N, s.Hkv, s.ks_t, s.ks_h, BN) ||
+      !make_tensor_map(&tmv, a.v, D, pk ? (int)n_tokens : s.N, s.Hkv, s.vs_t, s.vs_h, BN))
     return EI_ERR_CUDA;
   auto kern = sparse_attention_kernel<D, BN, NS, P_SMEM>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES) != cudaSuccess)
     return EI_ERR_CUDA;
-  const long long grid = (long long)s.H * s.C_S * (s.L_S / BM);
+  const long long grid = pk ? packed_grid : (long long)s.H * s.C_S * (s.L_S / BM);
   const float scale_log2 = a.scale * 1.4426950408889634f;
   kern<<<(unsigned)grid, ATT_THREADS, L::DYN_BYTES, st>>>(tmq, tmk, tmv, a.out, a.offsets, a.indices, a.status, s,
-                                                         scale_log2);
+                                                         scale_log2, pk, npk);
   return cudaGetLastError() == cudaSuccess ? EI_OK : EI_ERR_CUDA;
 }
 
 template <int D, int BN, int NSLOT>
-static int launch_pair_t(const Shape& s, const AttnArgs& a, cudaStream_t st) {
+static int launch_pair_t(const Shape& s, const AttnArgs& a, cudaStream_t st, const PackedSeq* pk = nullptr, int npk = 0,
+                         long long n_tokens = 0, long long packed_grid = 0) {
   using L = Att2Smem<D, BN, NSLOT>;
   static_assert(L::DYN_BYTES <= 232448, "shared memory budget exceeded");
   CUtensorMap tmq, tmk, tmv;
-  if (!make_tensor_map(&tmq, a.q, D, s.Nq, s.H, s.qs_t, s.qs_h, BM) ||
-      !make_tensor_map(&tmk, a.k, D, s.N, s.Hkv, s.ks_t, s.ks_h, BN) ||
-      !make_tensor_map(&tmv, a.v, D, s.N, s.Hkv, s.vs_t, s.vs_h, BN))
+  if (!make_tensor_map(&tmq, a.q, D, pk ? (int)n_tokens : s.Nq, s.H, s.qs_t, s.qs_h, BM) ||
+      !make_tensor_map(&tmk, a.k, D, pk ? (int)n_tokens : s.N, s.Hkv, s.ks_t, s.ks_h, BN) ||
+      !make_tensor_map(&tmv, a.v, D, pk ? (int)n_tokens : s.N, s.Hkv, s.vs_t, s.vs_h, BN))
     return EI_ERR_CUDA;
   auto kern = sparse_attention_pair_kernel<D, BN, NSLOT>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES) != cudaSuccess)
     return EI_ERR_CUDA;
-  const long long grid = (long long)s.H * s.C_S * (s.L_S / (2 * BM));
+  const long long grid = pk ? packed_grid : (long long)s.H * s.C_S * (s.L_S / (2 * BM));
   const float scale_log2 = a.scale * 1.4426950408889634f;
   kern<<<(unsigned)grid, ATT2_THREADS, L::DYN_BYTES, st>>>(tmq, tmk, tmv, a.out, a.offsets, a.indices, a.status, s,
-                                                          scale_log2);
+                                                          scale_log2, pk, npk);
   return cudaGetLastError() == cudaSuccess ? EI_OK : EI_ERR_CUDA;
 }
 
@@ -1744,6 +1768,32 @@ static int launch_persistent_t(const Shape& s, const AttnArgs& a, cudaStream_t s
   kern<<<grid, ATT3_THREADS, L::DYN_BYTES, st>>>(tmq, tmk, tmv, a.out, a.offsets, a.indices, a.status, a.sched, s,
                                                scale_log2, a.skip_log2, (int)n_items);
   return cudaGetLastError() == cudaSuccess ? EI_OK : EI_ERR_CUDA;
+}
+
+// The sequences of a packed batch in one launch, by the kernel launch_attention would pick for each of them without
+// flags: the quad-layout kernel (d = 128, 128-wide blocks, segments a multiple of 256), else a two-tile kernel
+// (segments a multiple of 256), else the one-tile kernel.  pk_host[i].w_att (packed_fill_work) counts the CTAs of the
+// earlier sequences accordingly.
+int launch_attention_packed(const PackedSeq* pk, const PackedSeq* pk_host, int npk, long long n_tokens, const AttnArgs& a,
+                            cudaStream_t st) {
+  const Shape& s = pk_host[npk - 1].s;
+  const bool pairs = s.L_S % (2 * BM) == 0 && s.d != 256;
+  const long long grid = pk_host[npk - 1].w_att + (long long)s.H * s.C_S * (s.L_S / (pairs ? 2 * BM : BM));
+  if (pairs && s.d == 128 && s.L_B == 128) return launch_attention_quad_packed(pk, pk_host, npk, n_tokens, a, st);
+  if (s.d == 256) {
+    if (s.L_B == 128) return launch_t<256, 128, 1, false>(s, a, st, pk, npk, n_tokens, grid);
+    return launch_t<256, 64, 2, false>(s, a, st, pk, npk, n_tokens, grid);
+  }
+  if (pairs) {
+    if (s.d == 128 && s.L_B == 64) return launch_pair_t<128, 64, 6>(s, a, st, pk, npk, n_tokens, grid);
+    if (s.d == 64 && s.L_B == 128) return launch_pair_t<64, 128, 6>(s, a, st, pk, npk, n_tokens, grid);
+    if (s.d == 64 && s.L_B == 64) return launch_pair_t<64, 64, 6>(s, a, st, pk, npk, n_tokens, grid);
+  }
+  if (s.d == 128 && s.L_B == 128) return launch_t<128, 128, 3, false>(s, a, st, pk, npk, n_tokens, grid);
+  if (s.d == 128 && s.L_B == 64) return launch_t<128, 64, 4, false>(s, a, st, pk, npk, n_tokens, grid);
+  if (s.d == 64 && s.L_B == 128) return launch_t<64, 128, 4, false>(s, a, st, pk, npk, n_tokens, grid);
+  if (s.d == 64 && s.L_B == 64) return launch_t<64, 64, 4, false>(s, a, st, pk, npk, n_tokens, grid);
+  return EI_ERR_UNSUPPORTED_SHAPE;
 }
 
 int launch_attention(const Shape& s, const AttnArgs& a, cudaStream_t st) {

@@ -314,7 +314,7 @@ sparse_attention_quad_kernel(const __grid_constant__ CUtensorMap tmq, const __gr
     s = P.s;
     bid -= P.w_att;
     tok0 = (int)P.tok0;
-    items += P.cell0 * pairs_per_seg * 8;
+    items += P.lcell0 * pairs_per_seg * 8;
     indices += P.idx0;
     out += P.tok0 * s.os_t;
   }

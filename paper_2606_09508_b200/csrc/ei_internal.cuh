@@ -39,11 +39,14 @@ __host__ __device__ inline int causal_blocks(const Shape& s, int i) {
 // were alone: the tables of the sequences lie one after another, each laid out exactly as a plan of that
 // sequence would lay them out.
 struct PackedSeq {
-  Shape s;
+  Shape s;           // the sequence's query-head shape
+  Shape ls;          // its list-head shape (H := H_kv under group-shared lists, else the same)
   long long tok0;   // first token of the sequence in q, k, v, out
-  long long cell0;  // first (head, segment) cell: entropy, multipliers, counts, query representatives, stage-4 records
-  long long off0;   // first entry of its offsets (cells + 1 entries per sequence)
-  long long sc0;    // first score
+  long long cell0;  // first (query head, segment) cell: entropy, query representatives
+  long long lcell0; // first (list head, segment) cell: group entropy, multipliers, counts, stage-4 records
+  long long off0;   // first entry of its offsets (list cells + 1 entries per sequence)
+  long long sc0;    // first score (per query head)
+  long long lsc0;   // first group score (per list head; = sc0 without group-shared lists)
   long long kb0;    // first key block in the K-representative arrays (KV-head stride there: the sequence's own C_B)
   long long idx0;   // first list entry
   long long T;      // TOTAL mode: the sequence's total
@@ -84,6 +87,9 @@ struct BudgetArgs;
 void packed_fill_work(PackedSeq* pk_host, int npk);  // fills w_pool, w_obs, w_sel, w_att
 cudaError_t launch_budget_packed(const PackedSeq* pk, int npk, const BudgetArgs& a, const float* entropy,
                                  unsigned char* rigid, int* Mfx, int* kblocks, int* offsets, Stats* stats, cudaStream_t st);
+// group-shared lists: the aggregation of every sequence's tables, one launch
+cudaError_t launch_group_aggregate_packed(const PackedSeq* pk, const PackedSeq* pk_host, int npk, const float* scores,
+                                          const float* entropy, float* g_scores, float* g_entropy, cudaStream_t st);
 cudaError_t launch_select_packed(const PackedSeq* pk, const PackedSeq* pk_host, int npk, const float* scores,
                                  const int* kblocks, const int* offsets, int* indices, int* items, cudaStream_t st);
 cudaError_t launch_pool(const Shape& s, const __nv_bfloat16* q, const __nv_bfloat16* k,
@@ -163,6 +169,9 @@ int launch_attention_tri(const Shape& s, const AttnArgs& a, cudaStream_t st);   
 // a.indices: the plan's arrays; offsets and shapes per sequence from pk)
 int launch_attention_quad_packed(const PackedSeq* pk, const PackedSeq* pk_host, int npk, long long n_tokens,
                                  const AttnArgs& a, cudaStream_t st);
+// any shape: picks the kernel launch_attention would pick without flags and launches it once over all sequences
+int launch_attention_packed(const PackedSeq* pk, const PackedSeq* pk_host, int npk, long long n_tokens, const AttnArgs& a,
+                            cudaStream_t st);
 // one record of 8 ints per (list cell, tile pair) from the plan's lists (ls: the list-head shape); a no-op for
 // shapes the tile-pair kernels do not take
 cudaError_t launch_attention_items(const Shape& ls, const int* offsets, const int* indices, int* items, cudaStream_t st);

@@ -788,7 +788,15 @@ cudaError_t launch_pool_observe(const Shape& s, const __nv_bfloat16* q, const __
 __global__ void __launch_bounds__(256) group_aggregate_kernel(Shape s, const float* __restrict__ scores,
                                                               const float* __restrict__ entropy,
                                                               float* __restrict__ g_scores,
-                                                              float* __restrict__ g_entropy) {
+                                                              float* __restrict__ g_entropy, const PackedSeq* pk) {
+  if (pk != nullptr) {  // a packed batch: blockIdx.y is my sequence
+    const PackedSeq& P = pk[blockIdx.y];
+    s = P.s;
+    scores += P.sc0;
+    entropy += P.cell0;
+    g_scores += P.lsc0;
+    g_entropy += P.lcell0;
+  }
   const long long n_sc = (long long)s.Hkv * s.SC, n_e = (long long)s.Hkv * s.C_S;
   const double inv_g = 1.0 / (double)s.G;
   for (long long x = (long long)blockIdx.x * 256 + threadIdx.x; x < n_sc + n_e; x += (long long)gridDim.x * 256) {
@@ -818,7 +826,20 @@ cudaError_t launch_group_aggregate(const Shape& s, const float* scores, const fl
   const long long n = (long long)s.Hkv * (s.SC + s.C_S);
   long long grid = (n + 255) / 256;
   if (grid > 148 * 8) grid = 148 * 8;
-  group_aggregate_kernel<<<(unsigned)grid, 256, 0, st>>>(s, scores, entropy, g_scores, g_entropy);
+  group_aggregate_kernel<<<(unsigned)grid, 256, 0, st>>>(s, scores, entropy, g_scores, g_entropy, nullptr);
+  return cudaGetLastError();
+}
+cudaError_t launch_group_aggregate_packed(const PackedSeq* pk, const PackedSeq* pk_host, int npk, const float* scores,
+                                          const float* entropy, float* g_scores, float* g_entropy, cudaStream_t st) {
+  long long nmax = 0;
+  for (int i = 0; i < npk; ++i) {
+    const Shape& s = pk_host[i].s;
+    const long long n = (long long)s.Hkv * (s.SC + s.C_S);
+    nmax = n > nmax ? n : nmax;
+  }
+  long long gx = (nmax + 255) / 256;
+  if (gx > 148 * 4) gx = 148 * 4;
+  group_aggregate_kernel<<<dim3((unsigned)gx, (unsigned)npk), 256, 0, st>>>(pk_host[0].s, scores, entropy, g_scores, g_entropy, pk);
   return cudaGetLastError();
 }
 
@@ -883,13 +904,13 @@ budget_kernel(Shape s, BudgetArgs a, const float* __restrict__ entropy, unsigned
               Stats* __restrict__ stats, const PackedSeq* pk) {
   if (pk != nullptr) {  // a packed batch: one CTA per sequence, each on its own share of the tables
     const PackedSeq& P = pk[blockIdx.x];
-    s = P.s;
+    s = P.ls;
     a.T = P.T;
     a.H_all = s.H;
-    entropy += P.cell0;
+    entropy += P.lcell0;
     rigid += P.head0;
-    Mfx += P.cell0;
-    kblocks += P.cell0;
+    Mfx += P.lcell0;
+    kblocks += P.lcell0;
     offsets += P.off0;
     stats += P.index;
   }
@@ -1110,13 +1131,13 @@ select_kernel(Shape s, const float* __restrict__ scores, const int* __restrict__
   int bid = blockIdx.x;
   if (pk != nullptr) {  // a packed batch: my sequence's shape, my CTA's number within it, its share of the tables
     const PackedSeq& P = pk[packed_find(pk, npk, bid, &PackedSeq::w_sel)];
-    s = P.s;
+    s = P.ls;
     bid -= P.w_sel;
-    scores += P.sc0;
-    kblocks += P.cell0;
+    scores += P.lsc0;
+    kblocks += P.lcell0;
     offsets += P.off0;
     indices += P.idx0;
-    if (items != nullptr) items += P.cell0 * pairs_per_seg * 8;
+    if (items != nullptr) items += P.lcell0 * pairs_per_seg * 8;
   }
   const long long c = (long long)bid * SEL_WARPS + warp;
   if (c >= s.cells) return;
@@ -1232,14 +1253,15 @@ void packed_fill_work(PackedSeq* pk_host, int npk) {
     pk_host[i].w_att = (int)wa;
     wp += s.cells + (long long)s.Hkv * s.C_B;
     wo += (long long)s.C_S * s.Hkv * nsub;
-    ws += (s.cells + SEL_WARPS - 1) / SEL_WARPS;
-    wa += (long long)s.H * s.C_S * (s.L_S / 256);
+    ws += (pk_host[i].ls.cells + SEL_WARPS - 1) / SEL_WARPS;
+    // stage 4: a CTA per tile pair where the two-tile kernels apply, else per 128-row tile
+    wa += (long long)s.H * s.C_S * ((s.L_S % 256 == 0 && s.d != 256) ? s.L_S / 256 : s.L_S / 128);
   }
 }
 
 cudaError_t launch_select_packed(const PackedSeq* pk, const PackedSeq* pk_host, int npk, const float* scores,
                                  const int* kblocks, const int* offsets, int* indices, int* items, cudaStream_t st) {
-  const Shape& s = pk_host[npk - 1].s;
+  const Shape& s = pk_host[npk - 1].ls;
   const unsigned grid = (unsigned)(pk_host[npk - 1].w_sel + (s.cells + SEL_WARPS - 1) / SEL_WARPS);
   const int pairs = s.L_S % 256 == 0 ? s.L_S / 256 : 0;
   select_kernel<<<grid, SEL_WARPS * 32, 0, st>>>(s, scores, kblocks, offsets, indices, pairs ? items : nullptr, pairs, pk, npk);

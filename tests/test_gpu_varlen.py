@@ -107,7 +107,7 @@ def test_packed_batch_arguments_are_checked():
     assert pl.status() == 0
 
 
-@pytest.mark.parametrize("mode", ["total", "base"])
+@pytest.mark.parametrize("mode", ["total", "base", "group"])
 @pytest.mark.parametrize("layout", ["head_major", "token_major"])
 def test_packed_batch_in_one_set_of_launches(mode, layout):
     # A plan made for the batch's total length has room for every sequence's tables side by side: the whole batch
@@ -116,11 +116,14 @@ def test_packed_batch_in_one_set_of_launches(mode, layout):
     rng = np.random.default_rng(7)
     if mode == "base":
         lens = [int(x) for x in rng.integers(130, 2100, size=11)] + [0, 2048, 129]
+    elif mode == "group":
+        lens = [int(x) for x in rng.integers(1700, 3000, size=5)] + [0, 2560]
     else:                                               # long enough that half the causal blocks cover the diagonal ones
         lens = [int(x) for x in rng.integers(1700, 3000, size=8)] + [0, 2048, 1701]
     total = sum(lens)
     q, k, v, (qd, kd, vd) = packed(layout, lens, seed=151)
-    fraction, base = (0.5, None) if mode == "total" else (0.0, 640.0)
+    fraction, base = (0.5, None) if mode != "base" else (0.0, 640.0)
+    flags = ei.FLAG_GROUP_SHARED if mode == "group" else 0
     # (room for every sequence's segments: each sequence rounds up to whole segments of its own)
     p = ei.params_default(H, HKV, D, sum(-(-n // L_S) * L_S for n in lens), L_S, L_B, fraction)
     if base is not None:
@@ -131,13 +134,14 @@ def test_packed_batch_in_one_set_of_launches(mode, layout):
         p.q_stride_head = p.k_stride_head = p.v_stride_head = p.o_stride_head = D
     else:
         p.q_stride_head = p.k_stride_head = p.v_stride_head = p.o_stride_head = total * D
+    p.flags = flags
     pl = ei.Plan(p)
     out = torch.full(qd.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
     cu = np.concatenate([[0], np.cumsum(lens)])
     n0 = pl.launches()
     pl.prefill_varlen(qd, kd, vd, out, cu)
     assert pl.status() == 0
-    assert pl.launches() - n0 == 5
+    assert pl.launches() - n0 == (6 if mode == "group" else 5)     # group-shared lists: one aggregation launch more
     got = to_bits(out)
     if layout == "token_major":
         got = np.ascontiguousarray(got.reshape(total, H, D).transpose(1, 0, 2))
@@ -150,6 +154,7 @@ def test_packed_batch_in_one_set_of_launches(mode, layout):
         p1 = ei.params_default(H, HKV, D, n, L_S, L_B, fraction)
         if base is not None:
             p1.base_budget_tokens = base
+        p1.flags = flags
         ref = ei.Plan(p1)
         o1 = torch.empty((H, n, D), dtype=torch.bfloat16, device="cuda")
         ref.plan(to_dev(qs), to_dev(ks))
@@ -158,3 +163,40 @@ def test_packed_batch_in_one_set_of_launches(mode, layout):
     with pytest.raises(ei.EiError) as e:                # the tables hold a batch now: nothing to attend from
         pl.sparse_prefill(qd, kd, vd, out)
     assert e.value.code == ei.STATUS["NOT_PLANNED"]
+
+
+@pytest.mark.parametrize("shape", [(4, 2, 64, 256, 64), (4, 2, 64, 256, 128), (6, 2, 128, 128, 64), (4, 1, 128, 384, 128),
+                                   (4, 2, 256, 256, 128), (2, 1, 256, 128, 64)],
+                         ids=lambda s_: "H%d_Hkv%d_d%d_LS%d_LB%d" % s_)
+def test_packed_batch_in_one_set_of_launches_other_shapes(shape):
+    # the same for the shapes that take the two-tile pair kernel (d or L_B = 64, segments a multiple of 256) and the
+    # one-tile kernel (other segment lengths, head_dim 256)
+    h, hkv, d, ls, lb = shape
+    rng = np.random.default_rng(11)
+    lens = [int(x) for x in rng.integers(70, 1500, size=7)] + [0, 4 * ls, ls + 1]
+    total = sum(lens)
+    q, k, v = synth.generate_plain(h, hkv, total, d, seed=152)
+    qd, kd, vd = to_dev(q), to_dev(k), to_dev(v)
+    p = ei.params_default(h, hkv, d, sum(-(-n // ls) * ls for n in lens), ls, lb, 0.0)
+    p.base_budget_tokens = 3.0 * lb
+    p.q_stride_head = p.k_stride_head = p.v_stride_head = p.o_stride_head = total * d
+    pl = ei.Plan(p)
+    out = torch.full(qd.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    n0 = pl.launches()
+    pl.prefill_varlen(qd, kd, vd, out, cu)
+    assert pl.status() == 0
+    assert pl.launches() - n0 == 5
+    got = to_bits(out).reshape(h, total, d)
+    for b, n in enumerate(lens):
+        if n == 0:
+            continue
+        lo, hi = int(cu[b]), int(cu[b + 1])
+        qs, ks, vs = (np.ascontiguousarray(a[:, lo:hi]) for a in (q, k, v))
+        p1 = ei.params_default(h, hkv, d, n, ls, lb, 0.0)
+        p1.base_budget_tokens = 3.0 * lb
+        ref = ei.Plan(p1)
+        o1 = torch.empty((h, n, d), dtype=torch.bfloat16, device="cuda")
+        ref.plan(to_dev(qs), to_dev(ks))
+        ref.sparse_prefill(to_dev(qs), to_dev(ks), to_dev(vs), o1)
+        np.testing.assert_array_equal(got[:, lo:hi], to_bits(o1).reshape(h, n, d), err_msg=f"sequence {b} of {n} tokens")
