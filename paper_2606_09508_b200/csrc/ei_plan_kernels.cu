@@ -898,6 +898,62 @@ __device__ long long block_excl_scan(long long v, long long* warp_sums, long lon
   return warp_sums[warp] + inc - v;
 }
 
+// class and multiplier recurrence of one head, by one warp (Alg. 3).  The division-heavy increments are computed
+// lane-parallel; only add / clamp is sequential.  Every lane carries the same running multiplier, so lane t keeps
+// the value after step t of its chunk.
+__device__ __forceinline__ void head_multipliers(const Shape& s, const BudgetArgs& a, const float* __restrict__ entropy,
+                                                 unsigned char* __restrict__ rigid, int* __restrict__ Mfx, int h, int lane,
+                                                 int* s_rigid) {
+    const float* e = entropy + (long long)h * s.C_S;
+    double emax = -INFINITY;
+    for (int i = lane; i < s.C_S; i += 32) emax = fmax(emax, (double)e[i]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) emax = fmax(emax, __shfl_xor_sync(0xffffffffu, emax, o));
+    const bool rg = emax < a.e_t;
+    if (lane == 0) {
+      rigid[h] = rg ? 1 : 0;
+      if (rg && s_rigid != nullptr) atomicAdd(s_rigid, 1);
+    }
+    int* Mh = Mfx + (long long)h * s.C_S;
+    const long long one_bits = __double_as_longlong(1.0), max_bits = __double_as_longlong(a.max_mult);
+    double m = 1.0;
+    for (int i0 = 0; i0 < s.C_S; i0 += 32) {
+      const int i = i0 + lane;
+      double inc = 0.0;
+      if (!rg && i >= 1 && i < s.C_S) {
+        const double prev = (double)e[i - 1], cur = (double)e[i];
+        const double den = fmax(prev, a.e_t);
+        const double fluct = __ddiv_rn(fabs(__dsub_rn(cur, prev)), den);
+        inc = __dmul_rn(a.alpha, __dsub_rn(fluct, a.delta_t));
+      }
+      double mine = 1.0;
+#pragma unroll
+      for (int t = 0; t < 32; ++t) {  // fixed trip count: the 32 broadcasts do not depend on the running value
+        const double inc_t = __shfl_sync(0xffffffffu, inc, t);
+        if (!rg && i0 + t >= 1 && i0 + t < s.C_S) {
+          // clamp to [1, max_mult] on the bit patterns: for non-NaN doubles a negative value has a negative
+          // pattern and non-negative values order like their patterns, so signed 64-bit compares give the same
+          // result as fmax / fmin with far less latency on the sequential chain
+          long long vb = __double_as_longlong(__dadd_rn(m, inc_t));
+          vb = vb < one_bits ? one_bits : vb;
+          vb = vb > max_bits ? max_bits : vb;
+          m = __longlong_as_double(vb);
+        }
+        if (t == lane) mine = m;
+      }
+      if (i < s.C_S) Mh[i] = (int)floor(__dadd_rn(__dmul_rn(mine, 4096.0), 0.5));
+    }
+}
+
+// The recurrences of the heads are independent and bound by the fp64 pipe of the SM they run on (a dependent
+// add per segment and head): spread over several CTAs, four heads each, they take a quarter of the time they
+// take inside the one-CTA budget kernel, which then runs the apportionment alone.
+__global__ void __launch_bounds__(128) multipliers_kernel(Shape s, BudgetArgs a, const float* __restrict__ entropy,
+                                                          unsigned char* __restrict__ rigid, int* __restrict__ Mfx) {
+  const int h = blockIdx.x * 4 + (threadIdx.x >> 5);
+  if (h < s.H) head_multipliers(s, a, entropy, rigid, Mfx, h, threadIdx.x & 31, nullptr);
+}
+
 __global__ void __launch_bounds__(BUD_THREADS, 1)
 budget_kernel(Shape s, BudgetArgs a, const float* __restrict__ entropy, unsigned char* __restrict__ rigid,
               int* __restrict__ Mfx, const int* Mall, int* __restrict__ kblocks, int* __restrict__ offsets,
@@ -932,49 +988,8 @@ budget_kernel(Shape s, BudgetArgs a, const float* __restrict__ entropy, unsigned
   }
 
   // ---- A: class + multiplier recurrence, one warp per head -------------------------------------------
-  // The division-heavy increments are computed lane-parallel; only add / clamp is sequential.  Every
-  // lane carries the same running multiplier, so lane t keeps the value after step t of its chunk.
-  for (int h = warp; h < s.H && a.phase != EI_BUDGET_PHASE_APPORTION; h += BUD_THREADS / 32) {
-    const float* e = entropy + (long long)h * s.C_S;
-    double emax = -INFINITY;
-    for (int i = lane; i < s.C_S; i += 32) emax = fmax(emax, (double)e[i]);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) emax = fmax(emax, __shfl_xor_sync(0xffffffffu, emax, o));
-    const bool rg = emax < a.e_t;
-    if (lane == 0) {
-      rigid[h] = rg ? 1 : 0;
-      if (rg) atomicAdd(&s_rigid, 1);
-    }
-    int* Mh = Mfx + (long long)h * s.C_S;
-    const long long one_bits = __double_as_longlong(1.0), max_bits = __double_as_longlong(a.max_mult);
-    double m = 1.0;
-    for (int i0 = 0; i0 < s.C_S; i0 += 32) {
-      const int i = i0 + lane;
-      double inc = 0.0;
-      if (!rg && i >= 1 && i < s.C_S) {
-        const double prev = (double)e[i - 1], cur = (double)e[i];
-        const double den = fmax(prev, a.e_t);
-        const double fluct = __ddiv_rn(fabs(__dsub_rn(cur, prev)), den);
-        inc = __dmul_rn(a.alpha, __dsub_rn(fluct, a.delta_t));
-      }
-      double mine = 1.0;
-#pragma unroll
-      for (int t = 0; t < 32; ++t) {  // fixed trip count: the 32 broadcasts do not depend on the running value
-        const double inc_t = __shfl_sync(0xffffffffu, inc, t);
-        if (!rg && i0 + t >= 1 && i0 + t < s.C_S) {
-          // clamp to [1, max_mult] on the bit patterns: for non-NaN doubles a negative value has a negative
-          // pattern and non-negative values order like their patterns, so signed 64-bit compares give the same
-          // result as fmax / fmin with far less latency on the sequential chain
-          long long vb = __double_as_longlong(__dadd_rn(m, inc_t));
-          vb = vb < one_bits ? one_bits : vb;
-          vb = vb > max_bits ? max_bits : vb;
-          m = __longlong_as_double(vb);
-        }
-        if (t == lane) mine = m;
-      }
-      if (i < s.C_S) Mh[i] = (int)floor(__dadd_rn(__dmul_rn(mine, 4096.0), 0.5));
-    }
-  }
+  for (int h = warp; h < s.H && a.phase != EI_BUDGET_PHASE_APPORTION; h += BUD_THREADS / 32)
+    head_multipliers(s, a, entropy, rigid, Mfx, h, lane, &s_rigid);
   __syncthreads();
   if (a.phase == EI_BUDGET_PHASE_MULTIPLIERS) return;  // (block-uniform)
   const int* Mt = a.phase == EI_BUDGET_PHASE_APPORTION ? Mall : Mfx;  // the table the apportionment runs over
@@ -991,7 +1006,10 @@ budget_kernel(Shape s, BudgetArgs a, const float* __restrict__ entropy, unsigned
     Mreg[t] = (c < c1) ? Mt[c] : 0;
     Creg[t] = (c < c1) ? causal_blocks(s, (i_first + t) % s.C_S) : 0;
   }
-  __shared__ int s_part[32];
+  __shared__ int s_acc[3];  // round r of the search adds into s_acc[r % 3]: one barrier per round (see below)
+  if (tid < 3) s_acc[tid] = 0;
+  __syncthreads();
+  int round = 0;
   // sum over all cells of k(c, b): every thread evaluates its own cells (from registers when they fit),
   // 32-bit partial sums (a thread's cells hold < 2^31 blocks; the total was checked to fit int32)
   auto block_total = [&](long long bcand) -> long long {
@@ -1012,14 +1030,15 @@ budget_kernel(Shape s, BudgetArgs a, const float* __restrict__ entropy, unsigned
     } else {
       for (int c = c0, i = i_first; c < c1; ++c, i = (i + 1 == s.C_S ? 0 : i + 1)) t += kc(Mt[c], causal_blocks(s, i));
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
-    __syncthreads();  // s_part free again
-    if (lane == 0) s_part[warp] = t;
+    // one warp-wide sum, one shared-memory add per warp, one barrier: the accumulator of round r + 2 was last read
+    // before the barrier of round r + 1, so thread 0 may clear it once this round's barrier has passed
+    t = __reduce_add_sync(0xffffffffu, t);
+    int* acc = &s_acc[round % 3];
+    if (lane == 0) atomicAdd(acc, t);
     __syncthreads();
-    int v = s_part[lane];
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    const int v = *reinterpret_cast<volatile int*>(acc);
+    if (tid == 0) s_acc[(round + 2) % 3] = 0;
+    ++round;
     return (long long)v;  // the same value in every thread
   };
   long long bstar;
@@ -1042,39 +1061,91 @@ budget_kernel(Shape s, BudgetArgs a, const float* __restrict__ entropy, unsigned
   }
 
   // ---- C: counts, leftover distribution, offsets ---------------------------------------------------
-  long long base_sum = 0, grow_cnt = 0;
-  for (int c = c0, i = i_first; c < c1; ++c, i = (i + 1 == s.C_S ? 0 : i + 1)) {
-    const int Ci = causal_blocks(s, i);
-    const long long k0 = cell_blocks(Mt[c], bstar, s.r, Ci);
-    base_sum += k0;
-    if (a.mode == EI_BUDGET_TOTAL_FRACTION) grow_cnt += cell_blocks(Mt[c], bstar + 1, s.r, Ci) > k0;
-  }
-  long long total0, dummy;
-  block_excl_scan(base_sum, s_warp, &total0);
-  long long R = 0;
-  if (a.mode == EI_BUDGET_TOTAL_FRACTION) R = a.T - total0;
-  long long grow_before = block_excl_scan(grow_cnt, s_warp, &dummy);
-  long long my_sum = 0;
+  long long R = 0, total1;
   int kmin = 0x7fffffff, kmax = 0;
-  for (int c = c0, i = i_first; c < c1; ++c, i = (i + 1 == s.C_S ? 0 : i + 1)) {
-    const int Ci = causal_blocks(s, i);
-    long long kc = cell_blocks(Mt[c], bstar, s.r, Ci);
-    if (a.mode == EI_BUDGET_TOTAL_FRACTION && cell_blocks(Mt[c], bstar + 1, s.r, Ci) > kc) {
-      if (grow_before < R) kc += 1;
-      grow_before += 1;
+  if (cpt <= CACHE) {
+    // every thread's cells are in registers: counts once, one scan for both the block sum (high word) and the
+    // number of cells that grow at b* + 1 (low word), one scan for the offsets
+    int kreg[CACHE];
+    unsigned grow = 0;
+    long long packed = 0;
+#pragma unroll
+    for (int u = 0; u < CACHE; ++u) {
+      kreg[u] = 0;
+      if (c0 + u < c1) {
+        const int k0 = cell_blocks(Mreg[u], bstar, s.r, Creg[u]);
+        kreg[u] = k0;
+        packed += (long long)k0 << 32;
+        if (a.mode == EI_BUDGET_TOTAL_FRACTION && cell_blocks(Mreg[u], bstar + 1, s.r, Creg[u]) > k0) {
+          grow |= 1u << u;
+          packed += 1;
+        }
+      }
     }
-    if (c >= cell_lo && c < cell_hi) {
-      kblocks[c - cell_lo] = (int)kc;
-      my_sum += kc;
-      kmin = min(kmin, (int)kc);
-      kmax = max(kmax, (int)kc);
+    long long tot;
+    const long long pre = block_excl_scan(packed, s_warp, &tot);
+    if (a.mode == EI_BUDGET_TOTAL_FRACTION) R = a.T - (tot >> 32);
+    long long grow_before = pre & 0xffffffffLL;
+    long long my_sum = 0;
+#pragma unroll
+    for (int u = 0; u < CACHE; ++u) {
+      const int c = c0 + u;
+      if (c < c1) {
+        if ((grow >> u) & 1u) {
+          if (grow_before < R) kreg[u] += 1;
+          grow_before += 1;
+        }
+        if (c >= cell_lo && c < cell_hi) {
+          kblocks[c - cell_lo] = kreg[u];
+          my_sum += kreg[u];
+          kmin = min(kmin, kreg[u]);
+          kmax = max(kmax, kreg[u]);
+        } else {
+          kreg[u] = 0;  // not mine: no share of the offsets
+        }
+      }
     }
-  }
-  long long total1;
-  long long off = block_excl_scan(my_sum, s_warp, &total1);
-  for (int c = max(c0, cell_lo); c < min(c1, cell_hi); ++c) {
-    offsets[c - cell_lo] = (int)off;
-    off += kblocks[c - cell_lo];
+    long long off = block_excl_scan(my_sum, s_warp, &total1);
+#pragma unroll
+    for (int u = 0; u < CACHE; ++u) {
+      const int c = c0 + u;
+      if (c < c1 && c >= cell_lo && c < cell_hi) {
+        offsets[c - cell_lo] = (int)off;
+        off += kreg[u];
+      }
+    }
+  } else {
+    long long base_sum = 0, grow_cnt = 0;
+    for (int c = c0, i = i_first; c < c1; ++c, i = (i + 1 == s.C_S ? 0 : i + 1)) {
+      const int Ci = causal_blocks(s, i);
+      const long long k0 = cell_blocks(Mt[c], bstar, s.r, Ci);
+      base_sum += k0;
+      if (a.mode == EI_BUDGET_TOTAL_FRACTION) grow_cnt += cell_blocks(Mt[c], bstar + 1, s.r, Ci) > k0;
+    }
+    long long total0, dummy;
+    block_excl_scan(base_sum, s_warp, &total0);
+    if (a.mode == EI_BUDGET_TOTAL_FRACTION) R = a.T - total0;
+    long long grow_before = block_excl_scan(grow_cnt, s_warp, &dummy);
+    long long my_sum = 0;
+    for (int c = c0, i = i_first; c < c1; ++c, i = (i + 1 == s.C_S ? 0 : i + 1)) {
+      const int Ci = causal_blocks(s, i);
+      long long kc = cell_blocks(Mt[c], bstar, s.r, Ci);
+      if (a.mode == EI_BUDGET_TOTAL_FRACTION && cell_blocks(Mt[c], bstar + 1, s.r, Ci) > kc) {
+        if (grow_before < R) kc += 1;
+        grow_before += 1;
+      }
+      if (c >= cell_lo && c < cell_hi) {
+        kblocks[c - cell_lo] = (int)kc;
+        my_sum += kc;
+        kmin = min(kmin, (int)kc);
+        kmax = max(kmax, (int)kc);
+      }
+    }
+    long long off = block_excl_scan(my_sum, s_warp, &total1);
+    for (int c = max(c0, cell_lo); c < min(c1, cell_hi); ++c) {
+      offsets[c - cell_lo] = (int)off;
+      off += kblocks[c - cell_lo];
+    }
   }
   if (kmax > 0) {
     atomicMin(&s_mink, kmin);
@@ -1096,6 +1167,14 @@ budget_kernel(Shape s, BudgetArgs a, const float* __restrict__ entropy, unsigned
 
 cudaError_t launch_budget(const Shape& s, const BudgetArgs& a, const float* entropy, unsigned char* rigid,
                           int* Mfx, const int* Mall, int* kblocks, int* offsets, Stats* stats, cudaStream_t st) {
+  if (a.phase != EI_BUDGET_PHASE_APPORTION && s.H >= 8) {  // the recurrences on their own, over several SMs
+    multipliers_kernel<<<(s.H + 3) / 4, 128, 0, st>>>(s, a, entropy, rigid, Mfx);
+    if (a.phase == EI_BUDGET_PHASE_MULTIPLIERS) return cudaGetLastError();
+    BudgetArgs b = a;
+    b.phase = EI_BUDGET_PHASE_APPORTION;
+    budget_kernel<<<1, BUD_THREADS, 0, st>>>(s, b, entropy, rigid, Mfx, Mfx, kblocks, offsets, stats, nullptr);
+    return cudaGetLastError();
+  }
   budget_kernel<<<1, BUD_THREADS, 0, st>>>(s, a, entropy, rigid, Mfx, Mall, kblocks, offsets, stats, nullptr);
   return cudaGetLastError();
 }
