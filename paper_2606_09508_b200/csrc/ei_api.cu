@@ -352,7 +352,8 @@ int run_budget(ei_plan_t* pl, int phase, const int* m_all, int n_heads_all, int 
   a.first_head = first_head;
   cudaError_t e = ei::launch_budget(pl->lshape, a, pl->group ? pl->g_entropy : pl->entropy, pl->rigid, pl->Mfx, m_all,
                                     pl->kblocks, pl->offsets, pl->stats, (cudaStream_t)stream);
-  pl->launches += 1;
+  // (with eight heads or more the whole stage is two kernels: the recurrences over several SMs, then the apportionment)
+  pl->launches += (phase == ei::EI_BUDGET_PHASE_ALL && pl->lshape.H >= 8) ? 2 : 1;
   return e == cudaSuccess ? EI_OK : EI_ERR_CUDA;
 }
 }  // namespace
